@@ -1,0 +1,373 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix (no GPU)."""
+import dataclasses
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import verillm_oracle as vo
+from paper_2509_24257_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def small_shape(n_layers=2, H=4, KV=2, dh=16, d=32, F=48, vocab=50):
+    return synth.ModelShape(n_layers, d, H, KV, dh, F, vocab, 10000.0, 1e-5)
+
+
+def random_model(shape, seed=0, std=0.2):
+    rng = np.random.default_rng(seed)
+    layers = []
+    for _ in range(shape.n_layers):
+        lw = {}
+        for name, shp in synth.layer_tensor_shapes(shape).items():
+            lw[name] = 1.0 + 0.1 * rng.standard_normal(shp) if name.endswith("norm") else std * rng.standard_normal(shp)
+        layers.append(lw)
+    embed = rng.standard_normal((shape.vocab, shape.d_model))
+    final = 1.0 + 0.1 * rng.standard_normal(shape.d_model)
+    return vo.make_model(shape, embed, final, layers)
+
+
+def test_prefill_equals_decode_position_by_position():
+    # the paper's core claim: one causal pass reproduces every decode-step state
+    shape = small_shape()
+    m = random_model(shape, 1)
+    toks = np.random.default_rng(2).integers(0, shape.vocab, 13)
+    a = vo.forward_prefill(m, toks)
+    b = vo.forward_decode_kvcache(m, toks, "f64")
+    assert a.shape == (shape.n_layers, 13, shape.d_model)
+    assert np.max(np.abs(a - b)) <= 1e-12 * np.max(np.abs(a))
+
+
+def test_causal_prefix_invariance():
+    shape = small_shape()
+    m = random_model(shape, 3)
+    toks = np.random.default_rng(4).integers(0, shape.vocab, 12)
+    base = vo.forward_prefill(m, toks)
+    other = toks.copy()
+    other[7] = (other[7] + 1) % shape.vocab
+    moved = vo.forward_prefill(m, other)
+    assert np.array_equal(base[:, :7], moved[:, :7])  # earlier positions bit-identical
+    assert np.max(np.abs(base[:, 7:] - moved[:, 7:])) > 1e-3  # position 7 and later do move
+    # a truncated sequence gives the same states on the shared prefix
+    short = vo.forward_prefill(m, toks[:9])
+    assert np.max(np.abs(short - base[:, :9])) <= 1e-13 * np.max(np.abs(base))
+
+
+def test_softmax_rows_sum_to_one_and_single_token_closed_form():
+    rng = np.random.default_rng(5)
+    T, H, KV, dh = 9, 4, 2, 8
+    q, k, v = rng.standard_normal((T, H, dh)), rng.standard_normal((T, KV, dh)), rng.standard_normal((T, KV, dh))
+    probs = []
+    out = vo.causal_attention(q, k, v, probs)
+    for w in probs:
+        assert np.max(np.abs(w.sum(axis=-1) - 1.0)) <= 1e-14
+        assert np.all(np.triu(w, 1) == 0.0)  # nothing attends to the future
+    # first position attends to itself only: output = v_0 of its KV head
+    for g in range(H):
+        assert np.array_equal(out[0, g], v[0, g * KV // H])
+    one = vo.causal_attention(q[:1], k[:1], v[:1])
+    assert np.array_equal(one[0, 3], v[0, 1])
+
+
+def test_attention_matches_library_sdpa():
+    rng = np.random.default_rng(6)
+    T, H, KV, dh = 17, 6, 2, 16
+    q, k, v = rng.standard_normal((T, H, dh)), rng.standard_normal((T, KV, dh)), rng.standard_normal((T, KV, dh))
+    ours = vo.causal_attention(q, k, v)
+    tq = torch.from_numpy(q).permute(1, 0, 2)[None]
+    tk = torch.from_numpy(k).permute(1, 0, 2)[None].repeat_interleave(H // KV, dim=1)
+    tv = torch.from_numpy(v).permute(1, 0, 2)[None].repeat_interleave(H // KV, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True)[0].permute(1, 0, 2).numpy()
+    assert np.max(np.abs(ours - ref)) <= 1e-12
+
+
+def test_rope_properties():
+    rng = np.random.default_rng(7)
+    dh = 32
+    q, k = rng.standard_normal((1, 1, dh)), rng.standard_normal((1, 1, dh))
+    base = 500000.0
+
+    def dot(m, n):
+        return float(np.sum(vo.rope(q, np.array([m]), base) * vo.rope(k, np.array([n]), base)))
+
+    assert abs(dot(5, 2) - dot(103, 100)) <= 1e-11  # depends on m - n only
+    assert abs(dot(40, 40) - dot(0, 0)) <= 1e-11
+    assert abs(dot(5, 2) - dot(2, 5)) > 1e-3  # and on its sign
+    assert np.array_equal(vo.rope(q, np.array([0]), base), q)  # identity at position 0
+    r = vo.rope(q, np.array([77]), base)
+    assert abs(np.linalg.norm(r) - np.linalg.norm(q)) <= 1e-13
+    # pairing (i, i + dh/2) and the frequency ladder, worked by hand for one pair
+    x = np.zeros((1, 1, dh))
+    x[0, 0, 3] = 1.0
+    y = vo.rope(x, np.array([10]), base)
+    ang = 10.0 * base ** (-2.0 * 3 / dh)
+    expect = np.zeros(dh)
+    expect[3], expect[3 + dh // 2] = np.cos(ang), np.sin(ang)
+    assert np.max(np.abs(y[0, 0] - expect)) <= 1e-15
+
+
+def test_rmsnorm_properties():
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal((5, 64)) * 3.0
+    g = np.ones(64)
+    y = vo.rmsnorm(x, g, 0.0)
+    assert np.max(np.abs(np.sqrt(np.mean(y * y, axis=-1)) - 1.0)) <= 1e-14
+    assert np.max(np.abs(vo.rmsnorm(7.5 * x, g, 0.0) - y)) <= 1e-14
+    g2 = 1.0 + rng.standard_normal(64)
+    assert np.max(np.abs(vo.rmsnorm(x, g2, 1e-5) - vo.rmsnorm(x, g, 1e-5) * g2)) <= 1e-14
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(x), (64,), torch.from_numpy(g2), 1e-5).numpy()
+    assert np.max(np.abs(vo.rmsnorm(x, g2, 1e-5) - ref)) <= 1e-13
+
+
+def test_gqa_equals_mha_with_replicated_kv_heads():
+    shape = small_shape(H=4, KV=2)
+    m = random_model(shape, 9)
+    rep = shape.n_heads // shape.n_kv_heads
+    mha_shape = dataclasses.replace(shape, n_kv_heads=shape.n_heads)
+    layers = []
+    for lw in m.layers:
+        lw2 = dict(lw)
+        for nm in ("wk", "wv"):
+            w = lw[nm].reshape(shape.n_kv_heads, shape.head_dim, shape.d_model)
+            lw2[nm] = np.repeat(w, rep, axis=0).reshape(shape.n_heads * shape.head_dim, shape.d_model)
+        layers.append(lw2)
+    m2 = vo.make_model(mha_shape, m.embed, m.final_norm, layers)
+    toks = np.random.default_rng(10).integers(0, shape.vocab, 11)
+    a, b = vo.forward_prefill(m, toks), vo.forward_prefill(m2, toks)
+    assert np.max(np.abs(a - b)) <= 1e-12 * np.max(np.abs(a))
+
+
+def test_zeroed_projection_closed_forms():
+    shape = small_shape()
+    m = random_model(shape, 11)
+    toks = np.random.default_rng(12).integers(0, shape.vocab, 9)
+    for lw in m.layers:
+        lw["wo"][:] = 0.0
+        lw["w_down"][:] = 0.0
+    st = vo.forward_prefill(m, toks)
+    for l in range(shape.n_layers):
+        assert np.array_equal(st[l], m.embed[toks])  # every block is the identity
+    m = random_model(shape, 11)
+    for lw in m.layers:
+        lw["w_gate"][:] = 0.0  # silu(0) = 0: the FFN adds nothing
+    st = vo.forward_prefill(m, toks)
+    h = m.embed[toks]
+    w = m.layers[0]
+    a = vo.rmsnorm(h, w["attn_norm"], m.rms_eps)
+    T = len(toks)
+    q = vo.rope((a @ w["wq"].T).reshape(T, 4, 16), np.arange(T), m.rope_base)
+    k = vo.rope((a @ w["wk"].T).reshape(T, 2, 16), np.arange(T), m.rope_base)
+    v = (a @ w["wv"].T).reshape(T, 2, 16)
+    u = h + vo.causal_attention(q, k, v).reshape(T, -1) @ w["wo"].T
+    assert np.max(np.abs(st[0] - u)) <= 1e-13
+
+
+def test_against_transformers_llama_float64():
+    """The whole forward against an independent library implementation of the architecture."""
+    from transformers import LlamaConfig, LlamaModel
+
+    shape = synth.ModelShape(3, 64, 4, 2, 16, 96, 101, 500000.0, 1e-5)
+    m = random_model(shape, 13, std=0.15)
+    cfg = LlamaConfig(
+        vocab_size=shape.vocab, hidden_size=shape.d_model, intermediate_size=shape.d_ffn,
+        num_hidden_layers=shape.n_layers, num_attention_heads=shape.n_heads,
+        num_key_value_heads=shape.n_kv_heads, head_dim=shape.head_dim, rms_norm_eps=shape.rms_eps,
+        rope_theta=shape.rope_base, attention_bias=False, mlp_bias=False, max_position_embeddings=256,
+        tie_word_embeddings=False,
+    )
+    hf = LlamaModel(cfg).double().eval()
+    sd = {"embed_tokens.weight": m.embed, "norm.weight": m.final_norm}
+    names = {"attn_norm": "input_layernorm", "wq": "self_attn.q_proj", "wk": "self_attn.k_proj",
+             "wv": "self_attn.v_proj", "wo": "self_attn.o_proj", "ffn_norm": "post_attention_layernorm",
+             "w_gate": "mlp.gate_proj", "w_up": "mlp.up_proj", "w_down": "mlp.down_proj"}
+    for l, lw in enumerate(m.layers):
+        for k, v in lw.items():
+            sd[f"layers.{l}.{names[k]}.weight"] = v
+    missing = hf.load_state_dict({k: torch.from_numpy(np.ascontiguousarray(v)) for k, v in sd.items()}, strict=False)
+    assert not [k for k in missing.missing_keys if "rotary" not in k]
+    toks = np.random.default_rng(14).integers(0, shape.vocab, 37)
+    with torch.no_grad():
+        out = hf(input_ids=torch.from_numpy(toks)[None], output_hidden_states=True, use_cache=False)
+    ours = vo.forward_prefill(m, toks)
+    for l in range(shape.n_layers - 1):
+        ref = out.hidden_states[l + 1][0].numpy()
+        assert np.linalg.norm(ours[l] - ref) <= 1e-5 * np.linalg.norm(ref), l
+    last = vo.rmsnorm(ours[-1], m.final_norm, m.rms_eps)  # the library applies the final norm to the last state
+    ref = out.last_hidden_state[0].numpy()
+    assert np.linalg.norm(last - ref) <= 1e-5 * np.linalg.norm(ref)
+
+
+def test_batch_independence_and_zero_deviation_accept():
+    shape = small_shape()
+    m = random_model(shape, 15)
+    rng = np.random.default_rng(16)
+    seqs = [rng.integers(0, shape.vocab, 10), rng.integers(0, shape.vocab, 7), rng.integers(0, shape.vocab, 12)]
+    check_seq = np.array([2, 0, 0, 2], dtype=np.int32)
+    check_pos = np.array([11, 3, 9, 0], dtype=np.int32)
+    own = np.stack([np.stack([vo.forward_prefill(m, seqs[s])[l, p] for s, p in zip(check_seq, check_pos)])
+                    for l in range(shape.n_layers)])
+    tol = vo.Tol(bit_aware=True)
+    rep = vo.verify_prefill(m, seqs, own, check_seq, check_pos, tol, "f32")
+    # against its own float64 states rounded to f32 the only deviation is that rounding
+    assert rep.pos_ok.tolist() == [1, 1, 1, 1] and rep.seq_ok.tolist() == [1, 1, 1]
+    assert rep.first_bad_layer.tolist() == [-1] * 4
+    assert np.max(rep.stats[..., vo.STAT_NAMES.index("rel_l2")]) == 0.0
+    assert rep.seq_score[1] == 0.0  # a sequence without checked positions: accepted, score 0
+    # order of sequences in the batch does not matter
+    rep2 = vo.verify_prefill(m, [seqs[2], seqs[1], seqs[0]], own, np.array([0, 2, 2, 0]), check_pos, tol, "f32")
+    assert np.array_equal(rep.stats, rep2.stats)
+    # prefix-only recomputation gives the same report
+    rep3 = vo.verify_prefill(m, seqs, own, check_seq, check_pos, tol, "f32", prefix_only=True)
+    assert np.max(np.abs(rep3.hidden - rep.hidden)) <= 1e-13 * np.max(np.abs(rep.hidden))
+
+
+def test_round_to_bf16_matches_library_conversion():
+    rng = np.random.default_rng(17)
+    x = np.concatenate([
+        rng.standard_normal(20000) * np.exp(rng.uniform(-60, 60, 20000)),
+        np.array([0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895313892515355e38, 1e-40, -1e-39, 65280.0, 65408.0]),
+    ]).astype(np.float32)  # float32 inputs: the library rounds float32 -> bf16 once
+    ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()
+    got = vo.round_to_bf16(x.astype(np.float64))
+    assert np.array_equal(ref, got)
+    bits = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(vo.widen_bf16_bits(bits), ref)
+    # ties go to even: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    assert vo.round_to_bf16(np.array([1.0 + 2.0 ** -8]))[0] == 1.0
+    assert vo.round_to_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+
+
+def test_compare_stats_hand_worked_vectors():
+    tol = vo.Tol(tau_large=0.25, e_w=1e-2, e_m=7)
+    u = 2.0 ** -7  # one bf16 step in [1, 2)
+    #            exact  +1 step  +8 steps  binade cross   other binade   tiny     sign flip
+    c = np.array([1.5, 1.5, 1.5, 1.0, 1.0, 0.0, 1.25])
+    h = np.array([1.5, 1.5 + u, 1.5 + 8 * u, 1.0 - u / 2, 0.5, 4e-6, -1.25])
+    s = dict(zip(vo.STAT_NAMES, vo.compare_stats(h, c, "bf16", tol)))
+    d = h - c
+    assert s["n_exact"] == 1 and s["n_nonfinite"] == 0
+    assert s["n_exp_mismatch"] == 3  # 1-u/2 (exp 126), 0.5 (exp 126), 4e-6 vs 0 (exp field 0)
+    assert s["p_e"] == 3 / 7
+    # mismatches: (1 - u/2) has mantissa 127 vs 0 -> large; 0.5 has mantissa 0 vs 0 -> small;
+    # 4e-6 = 1.0000110...b * 2^-18 rounds to mantissa 6 vs 0 -> small
+    assert s["n_mant_large"] == 1 and s["p_m"] == 1 / 3
+    # matches: exact (0 steps), +1 step (<= 1.28), +8 steps (large), sign flip (2*(128+32) steps, large)
+    assert s["n_mant_small"] == 2 and s["p_w"] == 2 / 4
+    assert s["max_abs"] == 2.5
+    assert abs(s["mae"] - np.sum(np.abs(d)) / 7) <= 1e-15
+    assert abs(s["mean_signed"] - np.sum(d) / 7) <= 1e-15
+    assert abs(s["rel_l2"] - np.linalg.norm(d) / np.linalg.norm(c)) <= 1e-15
+    assert s["q_small"] == 2 / 7  # the exact element and the 4e-6 one
+    assert s["z_large"] == 2 / 7  # |d| > 0.25: the 0.5 and the 2.5
+    # f32 serialisation: 23 mantissa bits, one bf16 step is 65536 f32 steps (<= 0.01 * 2^23 = 83886)
+    s32 = dict(zip(vo.STAT_NAMES, vo.compare_stats(h, c, "f32", tol)))
+    assert s32["n_mant_small"] == 2 and s32["n_exp_mismatch"] == 3
+    # non-finite values are counted and force a reject
+    hn = h.copy()
+    hn[2] = np.nan
+    sn = vo.compare_stats(hn, c, "bf16", tol)
+    assert sn[vo.STAT_NAMES.index("n_nonfinite")] == 1
+    assert not vo.layer_passes(sn, vo.Tol(rel_l2=0.0))
+    # reference of norm zero: relative error stays finite through the tiny floor
+    z = vo.compare_stats(np.array([1.0, 0.0]), np.array([0.0, 0.0]), "bf16", tol)
+    assert np.isfinite(z[0]) and z[0] > 1e20
+
+
+def test_threshold_directions():
+    tol = vo.Tol(rel_l2=0.25, max_abs=0.5, mae=0.0)
+    c = np.array([2.0, 0.0, 0.0, 0.0])
+    at = vo.compare_stats(np.array([2.5, 0.0, 0.0, 0.0]), c, "f32", tol)  # rel_l2 = 0.25, max_abs = 0.5 exactly
+    assert vo.layer_passes(at, tol)  # equality accepts
+    above = vo.compare_stats(np.array([2.5000001, 0.0, 0.0, 0.0]), c, "f32", tol)
+    assert not vo.layer_passes(above, tol)
+    # one bad layer rejects the position, one bad position rejects its sequence only
+    good = vo.compare_stats(c, c, "f32", tol)
+    stats = np.stack([np.stack([good, good, good]), np.stack([good, above, above]), np.stack([good, good, good])])
+    pos_ok, first_bad, seq_ok, score = vo.verdict(stats, np.array([0, 1, 1]), 3, tol)
+    assert pos_ok.tolist() == [1, 0, 1] and first_bad.tolist() == [-1, 1, -1]
+    assert seq_ok.tolist() == [1, 0, 1]
+    mae_bad = above[vo.STAT_NAMES.index("mae")]
+    assert abs(score[1] - (2 * mae_bad) / 6) <= 1e-15 and score[0] == 0.0 and score[2] == 0.0
+
+
+def _table_rows():
+    rows = []
+    for line in open(os.path.join(GOLDEN, "paper_table_bins.txt")):
+        if line.strip() and not line.startswith("#"):
+            rows.append([int(x) for x in line.split()])
+    return rows
+
+
+@pytest.mark.parametrize("row", _table_rows())
+def test_bit_aware_bookkeeping_reproduces_paper_table_bins(row):
+    """Elements realising one printed table row must give back the row's ratios, and the paper's
+    off-chain thresholds must separate the honest table from the quantised one."""
+    table, n, exact, m_large, m_small, x_large, x_small = row
+    assert m_large + m_small + x_large + x_small == n and exact <= m_small
+    u = 2.0 ** -7
+    c, h = [], []
+    for i in range(exact):
+        c.append(1.5); h.append(1.5)
+    for i in range(m_small - exact):
+        c.append(1.5); h.append(1.5 + u * (1 if i % 2 else -1))
+    for i in range(m_large):
+        c.append(1.5); h.append(1.5 + 8 * u * (1 if i % 2 else -1))
+    for i in range(x_large):  # just across a binade boundary: mantissa fields 0 and 127
+        if i % 2:
+            c.append(1.0); h.append(1.0 - u / 2)
+        else:
+            c.append(1.0 - u / 2); h.append(1.0)
+    for i in range(x_small):  # a factor of two apart: equal mantissa fields
+        if i % 2:
+            c.append(1.0); h.append(0.5)
+        else:
+            c.append(0.5); h.append(1.0)
+    perm = np.random.default_rng(n).permutation(n)
+    c, h = np.array(c)[perm], np.array(h)[perm]
+    tol = vo.Tol(rel_l2=0.0, bit_aware=True)  # the paper's off-chain thresholds are the defaults
+    st = vo.compare_stats(h, c, "bf16", tol)
+    s = dict(zip(vo.STAT_NAMES, st))
+    assert s["n_exact"] == exact
+    assert s["p_e"] == (x_large + x_small) / n
+    assert s["p_m"] == x_large / (x_large + x_small)
+    assert s["p_w"] == m_small / (m_large + m_small)
+    accept = bool(vo.layer_passes(st, tol))
+    if table == 2:
+        assert s["p_e"] > 0.05 and not accept  # quantised prover: rejected on P_e alone
+    elif n == 256:
+        assert accept  # 9/256 < 0.05, 7/9 > 0.75, 201/247 > 0.80
+    else:
+        assert s["p_e"] < 0.05 and s["p_m"] < 0.75 and not accept  # 64-element row: 2/3 and 48/61 miss the paper's own cut
+
+
+def test_bf16_decode_trace_is_close_but_not_identical():
+    shape = small_shape(d=64, dh=16, H=4, KV=2, F=96)
+    m = random_model(shape, 18)
+    toks = np.random.default_rng(19).integers(0, shape.vocab, 16)
+    exact = vo.forward_prefill(m, toks)
+    noisy = vo.forward_decode_kvcache(m, toks, "bf16")
+    rel = np.linalg.norm(noisy - exact, axis=-1) / np.linalg.norm(exact, axis=-1)
+    assert 1e-5 < rel.max() < 2e-2
+
+
+def test_synth_generator_is_reproducible_and_distributed_as_stated():
+    wl = synth.WORKLOADS["tiny"]
+    a = synth.layer_weights(wl, 0)
+    b = synth.layer_weights(wl, 0)
+    assert all(torch.equal(a[k], b[k]) for k in a)
+    w32 = synth.layer_weights(wl, 0, dtype=torch.float32)
+    assert torch.equal(w32["wq"].to(torch.bfloat16), a["wq"])  # bf16 copy = RNE of the fp32 master
+    assert abs(float(w32["w_gate"].std()) - 0.02) < 5e-4 and abs(float(w32["w_gate"].mean())) < 2e-4
+    assert abs(float(w32["ffn_norm"].mean()) - 1.0) < 0.02
+    assert not torch.equal(a["wk"], a["wv"])
+    toks = synth.token_streams(wl)
+    assert toks.shape == (1, 64) and toks.min() >= 0 and toks.max() < 1024
+    big = synth.token_streams(synth.WORKLOADS["small"])
+    assert big.shape == (4, 512) and len(np.unique(big)) > 1900
+    cs, cp = synth.check_positions(synth.WORKLOADS["small"])
+    assert len(cs) == 20 and len(set(zip(cs.tolist(), cp.tolist()))) == 20
+    rows = synth.embed_weights(wl, rows=torch.tensor([5, 1000]))
+    full = synth.embed_weights(wl)
+    assert torch.equal(rows, full[[5, 1000]])
