@@ -1,0 +1,447 @@
+// bf16 GEMM on the fifth-generation tensor cores: C[M][N] = A[M][K] * B[N][K]^T with fp32 accumulation
+// in tensor memory, and the fused epilogues of the verifier's layer (rotary embedding, residual add,
+// SwiGLU, gather-and-compare).  These are the projections inside F_i of S_{i+1} = F_i(S_i; W_i).
+//
+// One persistent CTA per SM walks a list of 128 x 256 output tiles.  Warp 0 feeds a 4-stage ring of
+// shared-memory tiles with TMA (128-byte swizzle), warp 1 issues tcgen05.mma (one thread) into one of
+// two 256-column TMEM accumulators, warps 2-5 drain the other accumulator (tcgen05.ld, one output row
+// per thread) and run the epilogue, so the epilogue of a tile overlaps the main loop of the next.
+// Every mbarrier wait is bounded; a wait that runs out records VERILLM_DEV_WAIT_TIMEOUT and the CTA
+// falls through to its tail, which frees the tensor memory.
+#include "kernels.h"
+
+namespace vl {
+
+namespace {
+
+constexpr int BM = kGemmBM, BN = kGemmBN, BK = kGemmBK;
+constexpr int STAGES = 4;
+constexpr int UMMA_K = 16;
+constexpr int A_STAGE_BYTES = BM * BK * 2;  // 16 KiB
+constexpr int B_STAGE_BYTES = BN * BK * 2;  // 32 KiB
+constexpr int TILE_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);
+constexpr int BAR_BYTES = 256;
+constexpr int GEMM_SMEM = TILE_BYTES + BAR_BYTES + 1024;  // + slack for the 1024-byte alignment
+constexpr int GEMM_THREADS = 192;
+constexpr int TMEM_COLS = 512;  // two fp32 accumulators of 128 lanes x 256 columns
+constexpr int GROUP_M = 16;     // tiles are walked in bands of 16 tile-rows, row index fastest
+
+struct TileCoord {
+    int m_idx, n_idx;
+};
+
+__device__ __forceinline__ TileCoord tile_coord(int tile, int num_m, int num_n) {
+    const int per_group = GROUP_M * num_n;
+    const int g = tile / per_group;
+    const int r = tile - g * per_group;
+    const int m_first = g * GROUP_M;
+    const int gm = min(GROUP_M, num_m - m_first);
+    TileCoord c;
+    c.n_idx = r / gm;
+    c.m_idx = m_first + (r - c.n_idx * gm);
+    return c;
+}
+
+__device__ __forceinline__ float silu_f(float z) { return z / (1.f + __expf(-z)); }
+
+// Stores 32 consecutive fp32 accumulators of one row as bf16 (64 bytes, 16-byte vectors).
+__device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&v)[32]) {
+    uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint4 u;
+        u.x = pack_bf16(v[8 * i + 0], v[8 * i + 1]);
+        u.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
+        u.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
+        u.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
+        d4[i] = u;
+    }
+}
+
+__device__ __forceinline__ void load_acc(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    __syncwarp();  // tcgen05.ld is warp-collective: lanes that skipped a store rejoin here
+    tmem_ld32(taddr, r);
+    tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Epilogue of one tile for one thread (= one output row).  `trow` is the TMEM address of the thread's
+// lane at column 0 of the accumulator.  tcgen05.ld is warp-collective: every branch that contains one
+// is uniform across the warp (it depends on the tile only); row validity only predicates memory traffic.
+template <int EPI>
+__device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t trow, int row, int n0, int n_idx) {
+    const bool row_ok = row < p.M;
+
+    if constexpr (EPI == EPI_STORE_BF16 || EPI == EPI_STORE_F32 || EPI == EPI_RESID_ADD ||
+                  EPI == EPI_RESID_ADD_COMPARE) {
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            const int col = n0 + c * 32;
+            if (col >= p.N) break;
+            float v[32];
+            load_acc(trow + c * 32, v);
+            if (!row_ok) continue;
+            if constexpr (EPI == EPI_STORE_BF16) {
+                store_bf16x32(reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<size_t>(row) * p.ldo + col, v);
+            } else if constexpr (EPI == EPI_STORE_F32) {
+                float4* d4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) +
+                                                       static_cast<size_t>(row) * p.ldo + col);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            } else {
+                float4* d4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) +
+                                                       static_cast<size_t>(row) * p.ldo + col);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float4 r = d4[i];
+                    r.x += v[4 * i];
+                    r.y += v[4 * i + 1];
+                    r.z += v[4 * i + 2];
+                    r.w += v[4 * i + 3];
+                    d4[i] = r;
+                }
+            }
+        }
+    } else if constexpr (EPI == EPI_QKV_ROPE) {
+        // heads of head_dim columns; inside a rotated head column i pairs with i + head_dim/2
+        const int dh = p.head_dim;
+        const int half_chunks = dh / 64;  // 32-column chunks per half head: 1 (dh 64) or 2 (dh 128)
+        const int pos = row_ok ? p.pos_of_token[row] : 0;
+        __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<size_t>(row_ok ? row : 0) * p.ldo;
+#pragma unroll 1
+        for (int hb = 0; hb < BN; hb += dh) {
+            const int col0 = n0 + hb;
+            if (col0 >= p.N) break;
+            const bool rotate = col0 < p.rope_cols;
+#pragma unroll 1
+            for (int j = 0; j < half_chunks; ++j) {
+                float lo[32], hi[32];
+                load_acc(trow + hb + j * 32, lo);
+                load_acc(trow + hb + dh / 2 + j * 32, hi);
+                if (!row_ok) continue;
+                if (rotate) {
+                    const float2* cs = p.rope_cs + static_cast<size_t>(pos) * (dh / 2) + j * 32;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float2 t = __ldg(cs + i);
+                        const float a = lo[i], b = hi[i];
+                        lo[i] = a * t.x - b * t.y;
+                        hi[i] = b * t.x + a * t.y;
+                    }
+                }
+                store_bf16x32(orow + col0 + j * 32, lo);
+                store_bf16x32(orow + col0 + dh / 2 + j * 32, hi);
+            }
+        }
+    } else if constexpr (EPI == EPI_SWIGLU) {
+        // weight rows were interleaved in blocks of 128: tile columns [0,128) gate, [128,256) up
+        __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<size_t>(row_ok ? row : 0) * p.ldo +
+                              static_cast<size_t>(n_idx) * (BN / 2);
+        if (n0 < p.N) {
+#pragma unroll 1
+            for (int c = 0; c < BN / 64; ++c) {
+                float g[32], u[32];
+                load_acc(trow + c * 32, g);
+                load_acc(trow + BN / 2 + c * 32, u);
+                if (!row_ok) continue;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) g[i] = silu_f(g[i]) * u[i];
+                store_bf16x32(orow + c * 32, g);
+            }
+        }
+    }
+}
+
+// Gather-and-compare on the rows of this tile that carry check slots: the thread re-reads the 256
+// residual values it has just written, streams the committed values of each slot on the row
+// (16-byte loads) and leaves one partial record per (slot, column tile).
+__device__ __forceinline__ void compare_row(const GemmParams& p, int row, int n0, int n_idx, int n_tiles) {
+    int slot = p.slot_first[row];
+    const int ncols = min(BN, p.N - n0);
+    const float* hrow = reinterpret_cast<const float*>(p.out) + static_cast<size_t>(row) * p.ldo + n0;
+#pragma unroll 1
+    for (int it = 0; slot >= 0 && it < p.n_check; ++it) {
+        CmpAcc acc;
+        acc.clear();
+        float* hout = p.hidden_out ? p.hidden_out + static_cast<size_t>(slot) * p.N + n0 : nullptr;
+        if (p.committed == nullptr) {
+            // gather only (trace generation): copy the row segment, no statistics
+            if (hout)
+                for (int j = 0; j < ncols; j += 4)
+                    *reinterpret_cast<float4*>(hout + j) = *reinterpret_cast<const float4*>(hrow + j);
+            slot = p.slot_next[slot];
+            continue;
+        }
+        if (p.cmp.commit_dtype == VERILLM_BF16) {
+            const uint4* c4 = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.committed) +
+                                                             static_cast<size_t>(slot) * p.N + n0);
+#pragma unroll 1
+            for (int j = 0; j < ncols; j += 8) {
+                const uint4 cv = __ldg(c4 + j / 8);
+                const float4 h0 = *reinterpret_cast<const float4*>(hrow + j);
+                const float4 h1 = *reinterpret_cast<const float4*>(hrow + j + 4);
+                acc.add(h0.x, cv.x << 16, p.cmp);
+                acc.add(h0.y, cv.x & 0xFFFF0000u, p.cmp);
+                acc.add(h0.z, cv.y << 16, p.cmp);
+                acc.add(h0.w, cv.y & 0xFFFF0000u, p.cmp);
+                acc.add(h1.x, cv.z << 16, p.cmp);
+                acc.add(h1.y, cv.z & 0xFFFF0000u, p.cmp);
+                acc.add(h1.z, cv.w << 16, p.cmp);
+                acc.add(h1.w, cv.w & 0xFFFF0000u, p.cmp);
+                if (hout) {
+                    *reinterpret_cast<float4*>(hout + j) = h0;
+                    *reinterpret_cast<float4*>(hout + j + 4) = h1;
+                }
+            }
+        } else {
+            const uint4* c4 = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(p.committed) +
+                                                             static_cast<size_t>(slot) * p.N + n0);
+#pragma unroll 1
+            for (int j = 0; j < ncols; j += 4) {
+                const uint4 cv = __ldg(c4 + j / 4);
+                const float4 h0 = *reinterpret_cast<const float4*>(hrow + j);
+                acc.add(h0.x, cv.x, p.cmp);
+                acc.add(h0.y, cv.y, p.cmp);
+                acc.add(h0.z, cv.z, p.cmp);
+                acc.add(h0.w, cv.w, p.cmp);
+                if (hout) *reinterpret_cast<float4*>(hout + j) = h0;
+            }
+        }
+        acc.store(p.partials + (static_cast<size_t>(slot) * n_tiles + n_idx) * kNPart);
+        slot = p.slot_next[slot];
+    }
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                  const __grid_constant__ GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
+    const uint32_t a_base = base;
+    const uint32_t b_base = base + STAGES * A_STAGE_BYTES;
+    const uint32_t bar_base = base + TILE_BYTES;
+    // barrier words (8 bytes each): full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
+    volatile uint32_t* tmem_slot_ptr =
+        reinterpret_cast<volatile uint32_t*>(smem_raw + (base - raw) + TILE_BYTES + 8 * (2 * STAGES + 4));
+    __shared__ int s_failed;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_m = (p.M + BM - 1) / BM;
+    const int num_n = (p.N + BN - 1) / BN;
+    const int num_tiles = num_m * num_n;
+    const int num_kb = (p.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        s_failed = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(acc_full_bar(a), 1);
+            mbar_init(acc_empty_bar(a), 4);  // one arrival per epilogue warp
+        }
+        fence_mbar_init();
+        tma_prefetch_desc(&tmap_a);
+        tma_prefetch_desc(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_ptr;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const TileCoord tc = tile_coord(tile, num_m, num_n);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    mbar_arrive_expect_tx(full_bar(stage), A_STAGE_BYTES + B_STAGE_BYTES);
+                    tma_load_2d(a_base + stage * A_STAGE_BYTES, &tmap_a, kb * BK, tc.m_idx * BM, full_bar(stage));
+                    tma_load_2d(b_base + stage * B_STAGE_BYTES, &tmap_b, kb * BK, tc.n_idx * BN, full_bar(stage));
+                    if (++stage == STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+            if (!ok) s_failed = 1;
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, p.status)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t a_desc = umma_desc_k_sw128(a_base + stage * A_STAGE_BYTES);
+                    const uint64_t b_desc = umma_desc_k_sw128(b_base + stage * B_STAGE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte units
+                        umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(stage));  // the stage is free once these MMAs have read it
+                    if (++stage == STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit(acc_full_bar(acc));
+                acc ^= 1;
+                if (acc == 0) acc_phase ^= 1u;
+            }
+            if (!ok) s_failed = 1;
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps 2..5
+        const int quarter = warp & 3;  // the TMEM lane quarter this warp may read
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            const TileCoord tc = tile_coord(tile, num_m, num_n);
+            if (!mbar_wait(acc_full_bar(acc), acc_phase, p.status)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const int row = tc.m_idx * BM + quarter * 32 + lane;
+            const int n0 = tc.n_idx * BN;
+            const uint32_t trow = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
+            epilogue_tile<EPI>(p, trow, row, n0, tc.n_idx);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar(acc));  // accumulator may be overwritten
+            if constexpr (EPI == EPI_RESID_ADD_COMPARE) {
+                if (row < p.M && p.slot_first != nullptr) compare_row(p, row, n0, tc.n_idx, num_n);
+                __syncwarp();
+            }
+            acc ^= 1;
+            if (acc == 0) acc_phase ^= 1u;
+        }
+        if (!ok) s_failed = 1;
+    }
+
+    // ---------------------------------------------------------------- tail
+    tc_fence_before();
+    __syncthreads();
+    if (s_failed) {
+        // a wait gave up: let copies and MMAs still in flight land before the CTA's memory goes away
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+template <int EPI>
+cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int num_sms,
+                       cudaStream_t stream) {
+    const int num_tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
+    if (num_tiles <= 0) return cudaSuccess;
+    const int grid = num_tiles < num_sms ? num_tiles : num_sms;
+    gemm_bf16_tcgen05<EPI><<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tb, p);
+    return cudaGetLastError();
+}
+
+template <int EPI>
+cudaError_t init_one() {
+    return cudaFuncSetAttribute(gemm_bf16_tcgen05<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+}  // namespace
+
+cudaError_t gemm_init() {
+    cudaError_t e;
+    if ((e = init_one<EPI_STORE_BF16>()) != cudaSuccess) return e;
+    if ((e = init_one<EPI_STORE_F32>()) != cudaSuccess) return e;
+    if ((e = init_one<EPI_QKV_ROPE>()) != cudaSuccess) return e;
+    if ((e = init_one<EPI_RESID_ADD>()) != cudaSuccess) return e;
+    if ((e = init_one<EPI_SWIGLU>()) != cudaSuccess) return e;
+    if ((e = init_one<EPI_RESID_ADD_COMPARE>()) != cudaSuccess) return e;
+    if (!g_encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return e;
+        if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
+        g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    return cudaSuccess;
+}
+
+int make_tmap_bf16_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld_elems,
+                      uint32_t box_rows) {
+    if (!g_encode) return -1;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0 || (ld_elems * 2) % 16 != 0) return -2;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {ld_elems * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : -3;
+}
+
+cudaError_t launch_gemm(int epilogue, const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int num_sms,
+                        cudaStream_t stream) {
+    switch (epilogue) {
+        case EPI_STORE_BF16: return launch_one<EPI_STORE_BF16>(ta, tb, p, num_sms, stream);
+        case EPI_STORE_F32: return launch_one<EPI_STORE_F32>(ta, tb, p, num_sms, stream);
+        case EPI_QKV_ROPE: return launch_one<EPI_QKV_ROPE>(ta, tb, p, num_sms, stream);
+        case EPI_RESID_ADD: return launch_one<EPI_RESID_ADD>(ta, tb, p, num_sms, stream);
+        case EPI_SWIGLU: return launch_one<EPI_SWIGLU>(ta, tb, p, num_sms, stream);
+        case EPI_RESID_ADD_COMPARE: return launch_one<EPI_RESID_ADD_COMPARE>(ta, tb, p, num_sms, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace vl

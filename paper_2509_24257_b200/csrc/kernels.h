@@ -1,0 +1,98 @@
+// Host-side launch interface between the C-ABI driver and the kernel translation units.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "compare.cuh"
+
+namespace vl {
+
+// ------------------------------------------------------------------ tensor-core GEMM
+enum GemmEpilogue {
+    EPI_STORE_BF16 = 0,      // C bf16
+    EPI_STORE_F32 = 1,       // C fp32
+    EPI_QKV_ROPE = 2,        // C bf16, rotary embedding on the q and k head columns
+    EPI_RESID_ADD = 3,       // resid fp32 += acc (in place)
+    EPI_SWIGLU = 4,          // tile holds 128 gate columns then 128 up columns: out bf16 = silu(g) * u
+    EPI_RESID_ADD_COMPARE = 5  // resid += acc, then gather-and-compare on the checked rows
+};
+
+constexpr int kGemmBM = 128;
+constexpr int kGemmBN = 256;
+constexpr int kGemmBK = 64;
+
+struct GemmParams {
+    int M, N, K;
+    void* out;  // bf16 / fp32 matrix or the fp32 residual stream
+    int ldo;    // leading dimension of out, elements
+    // EPI_QKV_ROPE
+    const float2* rope_cs;    // [position][head_dim/2] (cos, sin)
+    const int* pos_of_token;  // [M]
+    int head_dim;
+    int rope_cols;  // columns [0, rope_cols) hold heads that are rotated (q and k); the rest (v) are not
+    // EPI_RESID_ADD_COMPARE (slabs of the current layer)
+    const int* slot_first;  // [M] first check slot of a token row, -1 if none
+    const int* slot_next;   // [n_check] next slot on the same row, -1 terminates
+    int n_check;
+    const void* committed;  // [n_check][N]
+    float* partials;        // [n_check][n_tiles_n][kNPart]
+    float* hidden_out;      // optional [n_check][N]
+    CmpParams cmp;
+    int* status;
+};
+
+// Maps are encoded for a box of 64 (K) x 128 rows (A) and 64 x 256 rows (B), 128-byte swizzle.
+int make_tmap_bf16_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld_elems,
+                      uint32_t box_rows);
+cudaError_t launch_gemm(int epilogue, const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const GemmParams& p,
+                        int num_sms, cudaStream_t stream);
+cudaError_t gemm_init();  // raises the dynamic shared memory limit of every instantiation
+
+// ------------------------------------------------------------------ attention
+cudaError_t launch_attention(const void* qkv, const int* cu_seqlens_dev, int batch, int max_seqlen, int n_heads,
+                             int n_kv_heads, int head_dim, void* out, cudaStream_t stream);
+cudaError_t attention_init();
+
+// ------------------------------------------------------------------ small kernels
+cudaError_t launch_token_maps(const int* cu_seqlens_dev, int batch, int n_tokens, int* pos_of_token,
+                              int* seq_of_token, cudaStream_t stream);
+cudaError_t launch_slot_lists(const int* tok_of_slot, int n_check, int n_tokens, int* slot_first, int* slot_next,
+                              cudaStream_t stream);
+cudaError_t launch_embed(const int* tokens, const void* table, int n_tokens, int d_model, int vocab, float* resid,
+                         int* status, cudaStream_t stream);
+cudaError_t launch_rmsnorm(const float* x, const void* gain, void* y, int rows, int d, float eps,
+                           cudaStream_t stream);
+cudaError_t launch_compare_rows(const float* hidden, const void* committed, int n_rows, int d, const CmpParams& cmp,
+                                float* partials, cudaStream_t stream);
+struct TolDev {
+    float rel_l2, max_abs, mae, pe_max, pm_min, pw_min, e_abs_max, z_large_max, q_small_min;
+    int bit_aware;
+};
+// partials: [n_layers][n_check][n_tiles][kNPart] -> stats [n_check][n_layers][NSTAT], pos_ok, first_bad_layer
+cudaError_t launch_verdict(const float* partials, int n_layers, int n_check, int n_tiles, int d, const TolDev& tol,
+                           const int* status, float* stats, uint8_t* pos_ok, int* first_bad_layer,
+                           cudaStream_t stream);
+cudaError_t launch_seq_verdict(const float* stats, const uint8_t* pos_ok, const int* seq_of_slot, int n_check,
+                               int n_layers, int batch, uint8_t* seq_ok, float* seq_score, cudaStream_t stream);
+
+// ------------------------------------------------------------------ decode (prover side)
+// out[rows][n] (fp32) = x[rows][k] (bf16) * w[n][k]^T, rows <= 8 per launch group; optional in-place add.
+cudaError_t launch_skinny_gemm(const void* x, const void* w, float* out, int rows, int n, int k, int accumulate,
+                               cudaStream_t stream);
+cudaError_t launch_decode_rope_append(const float* qkv, const int* tok_index, const int* positions, int rows,
+                                      int n_heads, int n_kv_heads, int head_dim, const float2* rope_cs, void* q_out,
+                                      void* kv_cache_layer, cudaStream_t stream);
+cudaError_t launch_decode_attention(const void* q, const void* kv_cache_layer, const int* seq_start,
+                                    const int* positions, int rows, int n_heads, int n_kv_heads, int head_dim,
+                                    int max_keys, void* out, cudaStream_t stream);
+cudaError_t launch_swiglu_rows(const float* gu, void* out, int rows, int d_ffn, cudaStream_t stream);
+cudaError_t launch_gather_rows(const float* resid, const int* row_of_slot, const int* slots, int n_slots, int d,
+                               float* hidden_layer, cudaStream_t stream);
+cudaError_t launch_scatter_kv(const void* qkv, const int* dst_row, int rows, int n_heads, int n_kv_heads,
+                              int head_dim, void* kv_cache_layer, cudaStream_t stream);
+cudaError_t launch_convert_states(const float* src, void* dst, size_t n, int commit_dtype, cudaStream_t stream);
+cudaError_t launch_gather_tokens(const int* tokens, const int* src_index, int n, int* out, cudaStream_t stream);
+
+}  // namespace vl

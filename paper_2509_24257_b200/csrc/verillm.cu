@@ -1,0 +1,672 @@
+// C-ABI host driver: argument validation, weight re-layout, workspace planning and the launch
+// sequence of the verifier's prefill pass, the prover-side decode loop and the standalone comparison.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kernels.h"
+
+using namespace vl;
+
+namespace {
+
+typedef __nv_bfloat16 bf16;
+
+#define CU_TRY(expr)                                  \
+    do {                                              \
+        cudaError_t _e = (expr);                      \
+        if (_e != cudaSuccess) {                      \
+            g_last_cuda_error = _e;                   \
+            return _e == cudaErrorMemoryAllocation ? VERILLM_E_NOMEM : VERILLM_E_CUDA; \
+        }                                             \
+    } while (0)
+
+thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+
+struct LayerDev {
+    bf16 *attn_norm = nullptr, *ffn_norm = nullptr;
+    bf16 *wqkv = nullptr;  // [(H + 2 KV) dh][d]: q rows, k rows, v rows
+    bf16 *wo = nullptr;    // [d][H dh]
+    bf16 *wgu = nullptr;   // [2 F][d]: blocks of 128 gate rows followed by the 128 matching up rows
+    bf16 *wd = nullptr;    // [d][F]
+    CUtensorMap t_wqkv, t_wo, t_wgu, t_wd;
+};
+
+struct DecodeState {
+    bool ready = false;
+    bf16* kv_cache = nullptr;   // [n_layers][max_tokens][2 * KV * dh]
+    float* hidden_tmp = nullptr;  // [n_layers][max_checks][d]
+    float *resid = nullptr, *qkv = nullptr, *gu = nullptr;  // [max_batch][...]
+    bf16 *xn = nullptr, *q = nullptr, *attn = nullptr, *mid = nullptr;
+    int* ints = nullptr;  // index scratch: 6 * max_tokens + 3 * max_checks
+};
+
+}  // namespace
+
+struct verillm_model {
+    verillm_config cfg;
+    int device = 0, num_sms = 0;
+    int d_q = 0, d_kv = 0, n_qkv = 0, n_tiles_d = 0;
+    bf16 *embed = nullptr, *final_norm = nullptr;
+    std::vector<LayerDev> layers;
+    // workspace
+    float* resid = nullptr;
+    bf16 *xn = nullptr, *qkv = nullptr, *attn = nullptr, *mid = nullptr;
+    int *pos_of_token = nullptr, *seq_of_token = nullptr, *slot_first = nullptr, *slot_next = nullptr;
+    int *tok_of_slot = nullptr, *seq_of_slot = nullptr, *cu_dev = nullptr, *status = nullptr;
+    float* partials = nullptr;
+    float2* rope_cs = nullptr;
+    CUtensorMap t_xn, t_attn, t_mid;
+    DecodeState dec;
+    int last_launches = 0;
+};
+
+namespace {
+
+int ensure_init() {
+    static bool done[64] = {false};
+    int dev = 0;
+    CU_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return VERILLM_E_INVAL;
+    if (done[dev]) return VERILLM_OK;
+    cudaDeviceProp prop;
+    CU_TRY(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return VERILLM_E_ARCH;
+    CU_TRY(gemm_init());
+    CU_TRY(attention_init());
+    done[dev] = true;
+    return VERILLM_OK;
+}
+
+template <typename T>
+int dev_alloc(T** p, size_t count) {
+    *p = nullptr;
+    if (count == 0) return VERILLM_OK;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
+    if (e != cudaSuccess) {
+        g_last_cuda_error = e;
+        cudaGetLastError();
+        return VERILLM_E_NOMEM;
+    }
+    return VERILLM_OK;
+}
+
+bool shape_ok(const verillm_config& c) {
+    if (c.n_layers < 1 || c.d_model < 64 || c.n_heads < 1 || c.n_kv_heads < 1 || c.d_ffn < 128 || c.vocab < 1) return false;
+    if (c.head_dim != 64 && c.head_dim != 128) return false;
+    if (c.d_model % 64 != 0 || c.d_ffn % 128 != 0 || c.n_heads % c.n_kv_heads != 0) return false;
+    if (c.max_tokens < 1 || c.max_checks < 0 || c.max_batch < 1) return false;
+    if (!(c.rope_base > 1.f) || !(c.rms_eps >= 0.f)) return false;
+    return true;
+}
+
+int copy_in(void* dst, const void* src, size_t bytes, int on_device) {
+    CU_TRY(cudaMemcpy(dst, src, bytes, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice));
+    return VERILLM_OK;
+}
+
+TolDev tol_dev(const verillm_tol& t) {
+    TolDev d;
+    d.rel_l2 = t.rel_l2; d.max_abs = t.max_abs; d.mae = t.mae;
+    d.pe_max = t.pe_max; d.pm_min = t.pm_min; d.pw_min = t.pw_min; d.e_abs_max = t.e_abs_max;
+    d.z_large_max = t.z_large_max; d.q_small_min = t.q_small_min;
+    d.bit_aware = (t.flags & VERILLM_TOL_BIT_AWARE) ? 1 : 0;
+    return d;
+}
+
+CmpParams cmp_params(const verillm_tol& t, int commit_dtype) {
+    CmpParams c;
+    c.commit_dtype = commit_dtype;
+    c.tau_large = t.tau_large;
+    c.thr_w = t.e_w * static_cast<float>(1 << (commit_dtype == VERILLM_BF16 ? 7 : 23));
+    c.e_m = t.e_m;
+    return c;
+}
+
+// Checks the packed batch description; fills n_tokens and max_len.
+int check_batch(const verillm_model* m, const int32_t* cu, int32_t batch, int* n_tokens, int* max_len) {
+    if (!cu || batch < 1) return VERILLM_E_INVAL;
+    if (batch > m->cfg.max_batch) return VERILLM_E_SHAPE;
+    if (cu[0] != 0) return VERILLM_E_RANGE;
+    int mx = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (cu[b + 1] < cu[b]) return VERILLM_E_RANGE;
+        mx = std::max(mx, cu[b + 1] - cu[b]);
+    }
+    if (cu[batch] < 1) return VERILLM_E_RANGE;
+    if (cu[batch] > m->cfg.max_tokens) return VERILLM_E_SHAPE;
+    *n_tokens = cu[batch];
+    *max_len = mx;
+    return VERILLM_OK;
+}
+
+int check_slots(const verillm_model* m, const int32_t* cu, int32_t batch, const int32_t* check_seq,
+                const int32_t* check_pos, int32_t n_check, std::vector<int>* tok_of_slot) {
+    if (n_check < 0) return VERILLM_E_INVAL;
+    if (n_check > m->cfg.max_checks) return VERILLM_E_SHAPE;
+    if (n_check > 0 && (!check_seq || !check_pos)) return VERILLM_E_INVAL;
+    tok_of_slot->resize(n_check);
+    for (int s = 0; s < n_check; ++s) {
+        const int b = check_seq[s], p = check_pos[s];
+        if (b < 0 || b >= batch) return VERILLM_E_RANGE;
+        if (p < 0 || p >= cu[b + 1] - cu[b]) return VERILLM_E_RANGE;
+        (*tok_of_slot)[s] = cu[b] + p;
+    }
+    return VERILLM_OK;
+}
+
+// One transformer block over M packed tokens, residual stream updated in place.  With cmp_layer set the
+// down projection runs the gather(-and-compare) epilogue.
+struct LayerRun {
+    int M, batch, max_len;
+    const int* cu_dev;
+    const GemmParams* cmp_layer;  // fields slot_first .. cmp, or nullptr
+};
+
+int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStream_t st, int* launches) {
+    const verillm_config& c = m->cfg;
+    const LayerDev& w = m->layers[l];
+    GemmParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.status = status;
+    p.M = r.M;
+
+    CU_TRY(launch_rmsnorm(m->resid, w.attn_norm, m->xn, r.M, c.d_model, c.rms_eps, st));
+    p.N = m->n_qkv; p.K = c.d_model; p.out = m->qkv; p.ldo = m->n_qkv;
+    p.rope_cs = m->rope_cs; p.pos_of_token = m->pos_of_token; p.head_dim = c.head_dim; p.rope_cols = m->d_q + m->d_kv;
+    CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, w.t_wqkv, p, m->num_sms, st));
+    CU_TRY(launch_attention(m->qkv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads, c.head_dim, m->attn, st));
+    p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
+    CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_attn, w.t_wo, p, m->num_sms, st));
+    CU_TRY(launch_rmsnorm(m->resid, w.ffn_norm, m->xn, r.M, c.d_model, c.rms_eps, st));
+    p.N = 2 * c.d_ffn; p.K = c.d_model; p.out = m->mid; p.ldo = c.d_ffn;
+    CU_TRY(launch_gemm(EPI_SWIGLU, m->t_xn, w.t_wgu, p, m->num_sms, st));
+    p.N = c.d_model; p.K = c.d_ffn; p.out = m->resid; p.ldo = c.d_model;
+    if (r.cmp_layer) {
+        p.slot_first = r.cmp_layer->slot_first; p.slot_next = r.cmp_layer->slot_next; p.n_check = r.cmp_layer->n_check;
+        p.committed = r.cmp_layer->committed; p.partials = r.cmp_layer->partials; p.hidden_out = r.cmp_layer->hidden_out;
+        p.cmp = r.cmp_layer->cmp;
+        CU_TRY(launch_gemm(EPI_RESID_ADD_COMPARE, m->t_mid, w.t_wd, p, m->num_sms, st));
+    } else {
+        CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_mid, w.t_wd, p, m->num_sms, st));
+    }
+    *launches += 7;
+    return VERILLM_OK;
+}
+
+int ensure_decode_state(verillm_model* m) {
+    if (m->dec.ready) return VERILLM_OK;
+    const verillm_config& c = m->cfg;
+    DecodeState& d = m->dec;
+    int rc;
+    const size_t B = c.max_batch;
+    if ((rc = dev_alloc(&d.kv_cache, static_cast<size_t>(c.n_layers) * c.max_tokens * 2 * m->d_kv))) return rc;
+    if ((rc = dev_alloc(&d.hidden_tmp, static_cast<size_t>(c.n_layers) * std::max(c.max_checks, 1) * c.d_model))) return rc;
+    if ((rc = dev_alloc(&d.resid, B * c.d_model))) return rc;
+    if ((rc = dev_alloc(&d.qkv, B * m->n_qkv))) return rc;
+    if ((rc = dev_alloc(&d.gu, B * 2 * c.d_ffn))) return rc;
+    if ((rc = dev_alloc(&d.xn, B * c.d_model))) return rc;
+    if ((rc = dev_alloc(&d.q, B * m->d_q))) return rc;
+    if ((rc = dev_alloc(&d.attn, B * m->d_q))) return rc;
+    if ((rc = dev_alloc(&d.mid, B * c.d_ffn))) return rc;
+    if ((rc = dev_alloc(&d.ints, static_cast<size_t>(6) * c.max_tokens + 3 * static_cast<size_t>(std::max(c.max_checks, 1))))) return rc;
+    d.ready = true;
+    return VERILLM_OK;
+}
+
+}  // namespace
+
+// =============================================================================== C ABI
+
+extern "C" {
+
+void verillm_default_tol(verillm_tol* t) {
+    if (!t) return;
+    t->rel_l2 = 5e-2f; t->max_abs = 0.f; t->mae = 0.f;
+    t->pe_max = 0.05f; t->pm_min = 0.75f; t->pw_min = 0.80f; t->e_abs_max = 0.01f;
+    t->e_w = 1e-2f; t->e_m = 7;
+    t->tau_large = 0.f; t->z_large_max = -1.f; t->q_small_min = 0.f;
+    t->flags = 0u;
+}
+
+const char* verillm_strerror(int code) {
+    switch (code) {
+        case VERILLM_OK: return "ok";
+        case VERILLM_E_INVAL: return "invalid argument";
+        case VERILLM_E_SHAPE: return "unsupported shape or larger than the handle was sized for";
+        case VERILLM_E_RANGE: return "index out of range";
+        case VERILLM_E_NOMEM: return "device allocation failed";
+        case VERILLM_E_CUDA: return cudaGetErrorString(g_last_cuda_error);
+        case VERILLM_E_ARCH: return "device is not compute capability 10.x (sm_100a kernels)";
+        default: return "unknown error";
+    }
+}
+
+void verillm_free(verillm_model* m) {
+    if (!m) return;
+    cudaFree(m->embed); cudaFree(m->final_norm);
+    for (LayerDev& w : m->layers) {
+        cudaFree(w.attn_norm); cudaFree(w.ffn_norm); cudaFree(w.wqkv); cudaFree(w.wo); cudaFree(w.wgu); cudaFree(w.wd);
+    }
+    cudaFree(m->resid); cudaFree(m->xn); cudaFree(m->qkv); cudaFree(m->attn); cudaFree(m->mid);
+    cudaFree(m->pos_of_token); cudaFree(m->seq_of_token); cudaFree(m->slot_first); cudaFree(m->slot_next);
+    cudaFree(m->tok_of_slot); cudaFree(m->seq_of_slot); cudaFree(m->cu_dev); cudaFree(m->status);
+    cudaFree(m->partials); cudaFree(m->rope_cs);
+    DecodeState& d = m->dec;
+    cudaFree(d.kv_cache); cudaFree(d.hidden_tmp); cudaFree(d.resid); cudaFree(d.qkv); cudaFree(d.gu);
+    cudaFree(d.xn); cudaFree(d.q); cudaFree(d.attn); cudaFree(d.mid); cudaFree(d.ints);
+    delete m;
+}
+
+int32_t verillm_last_launch_count(const verillm_model* m) { return m ? m->last_launches : 0; }
+
+int verillm_load_layer(verillm_model* m, int32_t layer, const verillm_layer_weights* w, int32_t on_device) {
+    if (!m || !w || layer < 0 || layer >= m->cfg.n_layers) return VERILLM_E_INVAL;
+    if (!w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo || !w->ffn_norm || !w->w_gate || !w->w_up || !w->w_down)
+        return VERILLM_E_INVAL;
+    const verillm_config& c = m->cfg;
+    LayerDev& L = m->layers[layer];
+    const size_t d = c.d_model, e = sizeof(bf16);
+    int rc;
+    if ((rc = copy_in(L.attn_norm, w->attn_norm, d * e, on_device))) return rc;
+    if ((rc = copy_in(L.ffn_norm, w->ffn_norm, d * e, on_device))) return rc;
+    if ((rc = copy_in(L.wqkv, w->wq, m->d_q * d * e, on_device))) return rc;
+    if ((rc = copy_in(L.wqkv + m->d_q * d, w->wk, m->d_kv * d * e, on_device))) return rc;
+    if ((rc = copy_in(L.wqkv + (m->d_q + m->d_kv) * d, w->wv, m->d_kv * d * e, on_device))) return rc;
+    if ((rc = copy_in(L.wo, w->wo, d * m->d_q * e, on_device))) return rc;
+    if ((rc = copy_in(L.wd, w->w_down, d * c.d_ffn * e, on_device))) return rc;
+    // gate/up rows interleaved in blocks of 128 so that one 256-column output tile holds matching columns
+    const cudaMemcpyKind kind = on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    const size_t blk = 128 * d * e;
+    CU_TRY(cudaMemcpy2D(L.wgu, 2 * blk, w->w_gate, blk, blk, c.d_ffn / 128, kind));
+    CU_TRY(cudaMemcpy2D(reinterpret_cast<char*>(L.wgu) + blk, 2 * blk, w->w_up, blk, blk, c.d_ffn / 128, kind));
+    CU_TRY(cudaDeviceSynchronize());
+    return VERILLM_OK;
+}
+
+int verillm_load_globals(verillm_model* m, const void* embed, const void* final_norm, int32_t on_device) {
+    if (!m || !embed) return VERILLM_E_INVAL;
+    int rc;
+    if ((rc = copy_in(m->embed, embed, static_cast<size_t>(m->cfg.vocab) * m->cfg.d_model * sizeof(bf16), on_device)))
+        return rc;
+    if (final_norm && (rc = copy_in(m->final_norm, final_norm, m->cfg.d_model * sizeof(bf16), on_device))) return rc;
+    CU_TRY(cudaDeviceSynchronize());
+    return VERILLM_OK;
+}
+
+int verillm_load_weights(const verillm_config* cfg, const verillm_weights* weights, verillm_model** out) {
+    if (!cfg || !out) return VERILLM_E_INVAL;
+    *out = nullptr;
+    if (!shape_ok(*cfg)) return VERILLM_E_SHAPE;
+    int rc = ensure_init();
+    if (rc) return rc;
+    verillm_model* m = new (std::nothrow) verillm_model();
+    if (!m) return VERILLM_E_NOMEM;
+    m->cfg = *cfg;
+    const verillm_config& c = m->cfg;
+    cudaGetDevice(&m->device);
+    cudaDeviceGetAttribute(&m->num_sms, cudaDevAttrMultiProcessorCount, m->device);
+    m->d_q = c.n_heads * c.head_dim;
+    m->d_kv = c.n_kv_heads * c.head_dim;
+    m->n_qkv = m->d_q + 2 * m->d_kv;
+    m->n_tiles_d = (c.d_model + kGemmBN - 1) / kGemmBN;
+    m->layers.resize(c.n_layers);
+    const size_t d = c.d_model, T = c.max_tokens, NC = std::max(c.max_checks, 1);
+
+#define TRY_RC(expr)            \
+    do {                        \
+        rc = (expr);            \
+        if (rc) {               \
+            verillm_free(m);    \
+            return rc;          \
+        }                       \
+    } while (0)
+
+    TRY_RC(dev_alloc(&m->embed, static_cast<size_t>(c.vocab) * d));
+    TRY_RC(dev_alloc(&m->final_norm, d));
+    for (LayerDev& L : m->layers) {
+        TRY_RC(dev_alloc(&L.attn_norm, d));
+        TRY_RC(dev_alloc(&L.ffn_norm, d));
+        TRY_RC(dev_alloc(&L.wqkv, static_cast<size_t>(m->n_qkv) * d));
+        TRY_RC(dev_alloc(&L.wo, d * m->d_q));
+        TRY_RC(dev_alloc(&L.wgu, static_cast<size_t>(2) * c.d_ffn * d));
+        TRY_RC(dev_alloc(&L.wd, d * c.d_ffn));
+    }
+    TRY_RC(dev_alloc(&m->resid, T * d));
+    TRY_RC(dev_alloc(&m->xn, T * d));
+    TRY_RC(dev_alloc(&m->qkv, T * m->n_qkv));
+    TRY_RC(dev_alloc(&m->attn, T * m->d_q));
+    TRY_RC(dev_alloc(&m->mid, T * c.d_ffn));
+    TRY_RC(dev_alloc(&m->pos_of_token, T));
+    TRY_RC(dev_alloc(&m->seq_of_token, T));
+    TRY_RC(dev_alloc(&m->slot_first, T));
+    TRY_RC(dev_alloc(&m->slot_next, NC));
+    TRY_RC(dev_alloc(&m->tok_of_slot, NC));
+    TRY_RC(dev_alloc(&m->seq_of_slot, NC));
+    TRY_RC(dev_alloc(&m->cu_dev, static_cast<size_t>(c.max_batch) + 1));
+    TRY_RC(dev_alloc(&m->status, 1));
+    TRY_RC(dev_alloc(&m->partials, static_cast<size_t>(c.n_layers) * NC * m->n_tiles_d * kNPart));
+    TRY_RC(dev_alloc(&m->rope_cs, T * (c.head_dim / 2)));
+
+    // rotary table: angle = pos * base^(-2i/dh), evaluated in double, stored as (cos, sin) float pairs
+    {
+        const int half = c.head_dim / 2;
+        std::vector<float2> tab(T * half);
+        std::vector<double> inv_freq(half);
+        for (int i = 0; i < half; ++i) inv_freq[i] = std::pow(static_cast<double>(c.rope_base), -2.0 * i / c.head_dim);
+        for (size_t p = 0; p < T; ++p)
+            for (int i = 0; i < half; ++i) {
+                const double a = static_cast<double>(p) * inv_freq[i];
+                tab[p * half + i] = make_float2(static_cast<float>(std::cos(a)), static_cast<float>(std::sin(a)));
+            }
+        cudaError_t e = cudaMemcpy(m->rope_cs, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            g_last_cuda_error = e;
+            verillm_free(m);
+            return VERILLM_E_CUDA;
+        }
+    }
+    // TMA descriptors: activations are A operands (box of 128 rows), weights B operands (box of 256 rows)
+    bool ok = true;
+    ok = ok && make_tmap_bf16_2d(&m->t_xn, m->xn, T, d, d, kGemmBM) == 0;
+    ok = ok && make_tmap_bf16_2d(&m->t_attn, m->attn, T, m->d_q, m->d_q, kGemmBM) == 0;
+    ok = ok && make_tmap_bf16_2d(&m->t_mid, m->mid, T, c.d_ffn, c.d_ffn, kGemmBM) == 0;
+    for (LayerDev& L : m->layers) {
+        ok = ok && make_tmap_bf16_2d(&L.t_wqkv, L.wqkv, m->n_qkv, d, d, kGemmBN) == 0;
+        ok = ok && make_tmap_bf16_2d(&L.t_wo, L.wo, d, m->d_q, m->d_q, kGemmBN) == 0;
+        ok = ok && make_tmap_bf16_2d(&L.t_wgu, L.wgu, 2 * static_cast<uint64_t>(c.d_ffn), d, d, kGemmBN) == 0;
+        ok = ok && make_tmap_bf16_2d(&L.t_wd, L.wd, d, c.d_ffn, c.d_ffn, kGemmBN) == 0;
+    }
+    if (!ok) {
+        verillm_free(m);
+        return VERILLM_E_CUDA;
+    }
+    if (weights) {
+        if (weights->embed) TRY_RC(verillm_load_globals(m, weights->embed, weights->final_norm, weights->on_device));
+        if (weights->layers)
+            for (int l = 0; l < c.n_layers; ++l) TRY_RC(verillm_load_layer(m, l, &weights->layers[l], weights->on_device));
+    }
+#undef TRY_RC
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        g_last_cuda_error = e;
+        verillm_free(m);
+        return VERILLM_E_CUDA;
+    }
+    *out = m;
+    return VERILLM_OK;
+}
+
+int verillm_verify_prefill(verillm_model* m, const int32_t* tokens, const int32_t* cu_seqlens, int32_t batch,
+                           const void* committed_hidden, int32_t commit_dtype, const int32_t* check_seq,
+                           const int32_t* check_pos, int32_t n_check, const verillm_tol* tol,
+                           const verillm_report* rep, void* cuda_stream) {
+    if (!m || !tokens || !tol || !rep) return VERILLM_E_INVAL;
+    if (commit_dtype != VERILLM_BF16 && commit_dtype != VERILLM_F32) return VERILLM_E_INVAL;
+    if (!rep->seq_ok || !rep->seq_score || !rep->status) return VERILLM_E_INVAL;
+    if (n_check > 0 && (!committed_hidden || !rep->stats || !rep->pos_ok || !rep->first_bad_layer)) return VERILLM_E_INVAL;
+    int M = 0, max_len = 0, rc;
+    if ((rc = check_batch(m, cu_seqlens, batch, &M, &max_len))) return rc;
+    std::vector<int> tok_of_slot;
+    if ((rc = check_slots(m, cu_seqlens, batch, check_seq, check_pos, n_check, &tok_of_slot))) return rc;
+
+    const verillm_config& c = m->cfg;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int launches = 0;
+    CU_TRY(cudaMemsetAsync(rep->status, 0, sizeof(int), st));
+    CU_TRY(cudaMemcpyAsync(m->cu_dev, cu_seqlens, sizeof(int) * (batch + 1), cudaMemcpyHostToDevice, st));
+    if (n_check > 0) {
+        CU_TRY(cudaMemcpyAsync(m->tok_of_slot, tok_of_slot.data(), sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(m->seq_of_slot, check_seq, sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+    }
+    CU_TRY(launch_token_maps(m->cu_dev, batch, M, m->pos_of_token, m->seq_of_token, st));
+    CU_TRY(launch_slot_lists(m->tok_of_slot, n_check, M, m->slot_first, m->slot_next, st));
+    CU_TRY(launch_embed(tokens, m->embed, M, c.d_model, c.vocab, m->resid, rep->status, st));
+    launches += 2 + (n_check > 0 ? 1 : 0);
+
+    const size_t e_commit = commit_dtype == VERILLM_BF16 ? 2 : 4;
+    GemmParams cl;
+    std::memset(&cl, 0, sizeof(cl));
+    cl.slot_first = m->slot_first; cl.slot_next = m->slot_next; cl.n_check = n_check;
+    cl.cmp = cmp_params(*tol, commit_dtype);
+    LayerRun run{M, batch, max_len, m->cu_dev, n_check > 0 ? &cl : nullptr};
+    for (int l = 0; l < c.n_layers; ++l) {
+        const size_t slab = static_cast<size_t>(l) * n_check;
+        cl.committed = reinterpret_cast<const char*>(committed_hidden) + slab * c.d_model * e_commit;
+        cl.partials = m->partials + slab * m->n_tiles_d * kNPart;
+        cl.hidden_out = rep->hidden_out ? rep->hidden_out + slab * c.d_model : nullptr;
+        if ((rc = run_layer(m, l, run, rep->status, st, &launches))) return rc;
+    }
+    CU_TRY(launch_verdict(m->partials, c.n_layers, n_check, m->n_tiles_d, c.d_model, tol_dev(*tol), rep->status,
+                          rep->stats, rep->pos_ok, rep->first_bad_layer, st));
+    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, m->seq_of_slot, n_check, c.n_layers, batch, rep->seq_ok,
+                              rep->seq_score, st));
+    launches += (n_check > 0 ? 1 : 0) + 1;
+    m->last_launches = launches;
+    return VERILLM_OK;
+}
+
+int verillm_compare(const float* hidden, const void* committed, int32_t commit_dtype, int32_t n_layers, int32_t n_check,
+                    int32_t d_model, const int32_t* check_seq, int32_t batch, const verillm_tol* tol,
+                    const verillm_report* rep, void* cuda_stream) {
+    if (!hidden || !committed || !check_seq || !tol || !rep) return VERILLM_E_INVAL;
+    if (commit_dtype != VERILLM_BF16 && commit_dtype != VERILLM_F32) return VERILLM_E_INVAL;
+    if (n_layers < 1 || n_check < 1 || batch < 1) return VERILLM_E_INVAL;
+    if (d_model < 8 || d_model % 8 != 0) return VERILLM_E_SHAPE;
+    if (!rep->stats || !rep->pos_ok || !rep->first_bad_layer || !rep->seq_ok || !rep->seq_score || !rep->status)
+        return VERILLM_E_INVAL;
+    for (int s = 0; s < n_check; ++s)
+        if (check_seq[s] < 0 || check_seq[s] >= batch) return VERILLM_E_RANGE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const size_t rows = static_cast<size_t>(n_layers) * n_check;
+    float* partials = nullptr;
+    int* seq_dev = nullptr;
+    CU_TRY(cudaMallocAsync(reinterpret_cast<void**>(&partials), rows * kNPart * sizeof(float), st));
+    CU_TRY(cudaMallocAsync(reinterpret_cast<void**>(&seq_dev), sizeof(int) * n_check, st));
+    CU_TRY(cudaMemsetAsync(rep->status, 0, sizeof(int), st));
+    CU_TRY(cudaMemcpyAsync(seq_dev, check_seq, sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+    CU_TRY(launch_compare_rows(hidden, committed, static_cast<int>(rows), d_model, cmp_params(*tol, commit_dtype), partials, st));
+    CU_TRY(launch_verdict(partials, n_layers, n_check, 1, d_model, tol_dev(*tol), rep->status, rep->stats, rep->pos_ok,
+                          rep->first_bad_layer, st));
+    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, seq_dev, n_check, n_layers, batch, rep->seq_ok, rep->seq_score, st));
+    CU_TRY(cudaFreeAsync(partials, st));
+    CU_TRY(cudaFreeAsync(seq_dev, st));
+    return VERILLM_OK;
+}
+
+int verillm_decode_commit(verillm_model* m, const int32_t* tokens, const int32_t* cu_seqlens, int32_t batch,
+                          int32_t n_prefill, const int32_t* check_seq, const int32_t* check_pos, int32_t n_check,
+                          void* committed_out, int32_t commit_dtype, int32_t* status, void* cuda_stream) {
+    if (!m || !tokens || n_prefill < 0) return VERILLM_E_INVAL;
+    if (commit_dtype != VERILLM_BF16 && commit_dtype != VERILLM_F32) return VERILLM_E_INVAL;
+    if (n_check > 0 && !committed_out) return VERILLM_E_INVAL;
+    int M = 0, max_len = 0, rc;
+    if ((rc = check_batch(m, cu_seqlens, batch, &M, &max_len))) return rc;
+    std::vector<int> tok_of_slot;
+    if ((rc = check_slots(m, cu_seqlens, batch, check_seq, check_pos, n_check, &tok_of_slot))) return rc;
+    if ((rc = ensure_decode_state(m))) return rc;
+
+    const verillm_config& c = m->cfg;
+    DecodeState& d = m->dec;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int* dev_status = status ? status : m->status;
+    CU_TRY(cudaMemsetAsync(dev_status, 0, sizeof(int), st));
+    const size_t T = c.max_tokens, NC = std::max(c.max_checks, 1);
+    // index scratch layout
+    int* i_src = d.ints;                 // [Mp] packed-prompt row -> token index in the full batch
+    int* i_tok = d.ints + T;             // gathered token ids (prompt rows, then one decode step)
+    int* i_row_tok = d.ints + 2 * T;     // per decode row: token index in the full batch
+    int* i_row_pos = d.ints + 3 * T;     // per decode row: position
+    int* i_row_start = d.ints + 4 * T;   // per decode row: first token index of its sequence
+    int* i_misc = d.ints + 5 * T;        // prompt-phase slot rows [NC] live in tok_of_slot; spare
+    int* i_slot_row = d.ints + 6 * T;    // [NC] per sorted slot: row inside its decode step
+    int* i_slot_id = i_slot_row + NC;    // [NC] per sorted slot: slot index
+    (void)i_misc;
+
+    // ---------------------------------------------------------------- phase A: parallel pass over the prompts
+    std::vector<int> cu_p(batch + 1, 0), np(batch);
+    for (int b = 0; b < batch; ++b) {
+        np[b] = std::min(n_prefill, cu_seqlens[b + 1] - cu_seqlens[b]);
+        cu_p[b + 1] = cu_p[b] + np[b];
+    }
+    const int Mp = cu_p[batch];
+    if (Mp > 0) {
+        std::vector<int> src(Mp), slot_row(n_check);
+        int max_np = 0;
+        for (int b = 0; b < batch; ++b) {
+            max_np = std::max(max_np, np[b]);
+            for (int p = 0; p < np[b]; ++p) src[cu_p[b] + p] = cu_seqlens[b] + p;
+        }
+        for (int s = 0; s < n_check; ++s)
+            slot_row[s] = check_pos[s] < np[check_seq[s]] ? cu_p[check_seq[s]] + check_pos[s] : -1;
+        CU_TRY(cudaMemcpyAsync(i_src, src.data(), sizeof(int) * Mp, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(m->cu_dev, cu_p.data(), sizeof(int) * (batch + 1), cudaMemcpyHostToDevice, st));
+        if (n_check > 0)
+            CU_TRY(cudaMemcpyAsync(m->tok_of_slot, slot_row.data(), sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+        CU_TRY(launch_gather_tokens(tokens, i_src, Mp, i_tok, st));
+        CU_TRY(launch_token_maps(m->cu_dev, batch, Mp, m->pos_of_token, m->seq_of_token, st));
+        CU_TRY(launch_slot_lists(m->tok_of_slot, n_check, Mp, m->slot_first, m->slot_next, st));
+        CU_TRY(launch_embed(i_tok, m->embed, Mp, c.d_model, c.vocab, m->resid, dev_status, st));
+        GemmParams cl;
+        std::memset(&cl, 0, sizeof(cl));
+        cl.slot_first = m->slot_first; cl.slot_next = m->slot_next; cl.n_check = n_check;
+        cl.committed = nullptr; cl.partials = nullptr;
+        LayerRun run{Mp, batch, max_np, m->cu_dev, n_check > 0 ? &cl : nullptr};
+        int launches = 0;
+        for (int l = 0; l < c.n_layers; ++l) {
+            cl.hidden_out = d.hidden_tmp + static_cast<size_t>(l) * n_check * c.d_model;
+            if ((rc = run_layer(m, l, run, dev_status, st, &launches))) return rc;
+            // run_layer leaves this layer's rotated keys and values in qkv: append them to the cache
+            CU_TRY(launch_scatter_kv(m->qkv, i_src, Mp, c.n_heads, c.n_kv_heads, c.head_dim,
+                                     d.kv_cache + static_cast<size_t>(l) * T * 2 * m->d_kv, st));
+        }
+    }
+
+    // ---------------------------------------------------------------- phase B: token-by-token decode
+    // rows of step t: the sequences with n_prefill <= t < len, in batch order
+    std::vector<int> step_first, row_tok, row_pos, row_start;
+    std::vector<std::vector<int>> row_of_seq_at;  // not stored: recomputed below
+    int t_begin = max_len, t_end = max_len;
+    for (int b = 0; b < batch; ++b) t_begin = std::min(t_begin, np[b]);
+    for (int t = t_begin; t < t_end; ++t) {
+        step_first.push_back(static_cast<int>(row_tok.size()));
+        for (int b = 0; b < batch; ++b) {
+            const int len = cu_seqlens[b + 1] - cu_seqlens[b];
+            if (t >= np[b] && t < len) {
+                row_tok.push_back(cu_seqlens[b] + t);
+                row_pos.push_back(t);
+                row_start.push_back(cu_seqlens[b]);
+            }
+        }
+    }
+    step_first.push_back(static_cast<int>(row_tok.size()));
+    const int n_rows_total = static_cast<int>(row_tok.size());
+    if (n_rows_total > 0) {
+        // check slots of decoded positions, grouped by step
+        std::vector<int> order;
+        for (int s = 0; s < n_check; ++s)
+            if (check_pos[s] >= np[check_seq[s]]) order.push_back(s);
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return check_pos[a] < check_pos[b]; });
+        std::vector<int> slot_row(order.size()), slot_id(order.size()), slots_first(t_end - t_begin + 1, 0);
+        {
+            size_t k = 0;
+            for (int t = t_begin; t < t_end; ++t) {
+                slots_first[t - t_begin] = static_cast<int>(k);
+                while (k < order.size() && check_pos[order[k]] == t) {
+                    const int s = order[k];
+                    int row = 0;  // rank of the slot's sequence among the rows of step t
+                    for (int b = 0; b < check_seq[s]; ++b) {
+                        const int len = cu_seqlens[b + 1] - cu_seqlens[b];
+                        if (t >= np[b] && t < len) ++row;
+                    }
+                    slot_row[k] = row;
+                    slot_id[k] = s;
+                    ++k;
+                }
+            }
+            slots_first[t_end - t_begin] = static_cast<int>(k);
+        }
+        CU_TRY(cudaMemcpyAsync(i_row_tok, row_tok.data(), sizeof(int) * n_rows_total, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(i_row_pos, row_pos.data(), sizeof(int) * n_rows_total, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(i_row_start, row_start.data(), sizeof(int) * n_rows_total, cudaMemcpyHostToDevice, st));
+        if (!order.empty()) {
+            CU_TRY(cudaMemcpyAsync(i_slot_row, slot_row.data(), sizeof(int) * order.size(), cudaMemcpyHostToDevice, st));
+            CU_TRY(cudaMemcpyAsync(i_slot_id, slot_id.data(), sizeof(int) * order.size(), cudaMemcpyHostToDevice, st));
+        }
+        for (int t = t_begin; t < t_end; ++t) {
+            const int r0 = step_first[t - t_begin], rows = step_first[t - t_begin + 1] - r0;
+            if (rows == 0) continue;
+            const int s0 = slots_first[t - t_begin], n_slots = slots_first[t - t_begin + 1] - s0;
+            CU_TRY(launch_gather_tokens(tokens, i_row_tok + r0, rows, i_tok, st));
+            CU_TRY(launch_embed(i_tok, m->embed, rows, c.d_model, c.vocab, d.resid, dev_status, st));
+            for (int l = 0; l < c.n_layers; ++l) {
+                const LayerDev& w = m->layers[l];
+                bf16* cache_l = d.kv_cache + static_cast<size_t>(l) * T * 2 * m->d_kv;
+                CU_TRY(launch_rmsnorm(d.resid, w.attn_norm, d.xn, rows, c.d_model, c.rms_eps, st));
+                CU_TRY(launch_skinny_gemm(d.xn, w.wqkv, d.qkv, rows, m->n_qkv, c.d_model, 0, st));
+                CU_TRY(launch_decode_rope_append(d.qkv, i_row_tok + r0, i_row_pos + r0, rows, c.n_heads, c.n_kv_heads,
+                                                 c.head_dim, m->rope_cs, d.q, cache_l, st));
+                CU_TRY(launch_decode_attention(d.q, cache_l, i_row_start + r0, i_row_pos + r0, rows, c.n_heads,
+                                               c.n_kv_heads, c.head_dim, t + 1, d.attn, st));
+                CU_TRY(launch_skinny_gemm(d.attn, w.wo, d.resid, rows, c.d_model, m->d_q, 1, st));
+                CU_TRY(launch_rmsnorm(d.resid, w.ffn_norm, d.xn, rows, c.d_model, c.rms_eps, st));
+                CU_TRY(launch_skinny_gemm(d.xn, w.wgu, d.gu, rows, 2 * c.d_ffn, c.d_model, 0, st));
+                CU_TRY(launch_swiglu_rows(d.gu, d.mid, rows, c.d_ffn, st));
+                CU_TRY(launch_skinny_gemm(d.mid, w.wd, d.resid, rows, c.d_model, c.d_ffn, 1, st));
+                if (n_slots > 0)
+                    CU_TRY(launch_gather_rows(d.resid, i_slot_row + s0, i_slot_id + s0, n_slots, c.d_model,
+                                              d.hidden_tmp + static_cast<size_t>(l) * n_check * c.d_model, st));
+            }
+        }
+    }
+    if (n_check > 0)
+        CU_TRY(launch_convert_states(d.hidden_tmp, committed_out, static_cast<size_t>(c.n_layers) * n_check * c.d_model,
+                                     commit_dtype, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    return VERILLM_OK;
+}
+
+int verillm_op_gemm(const void* a, const void* b, void* cmat, int32_t M, int32_t N, int32_t K, int32_t out_f32,
+                    int32_t* status, void* cuda_stream) {
+    if (!a || !b || !cmat || M < 1 || N < 1 || K < 1) return VERILLM_E_INVAL;
+    if (K % 8 != 0 || N % 32 != 0) return VERILLM_E_SHAPE;
+    int rc = ensure_init();
+    if (rc) return rc;
+    int dev = 0, sms = 0;
+    CU_TRY(cudaGetDevice(&dev));
+    CU_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CUtensorMap ta, tb;
+    if (make_tmap_bf16_2d(&ta, a, M, K, K, kGemmBM) != 0) return VERILLM_E_CUDA;
+    if (make_tmap_bf16_2d(&tb, b, N, K, K, kGemmBN) != 0) return VERILLM_E_CUDA;
+    GemmParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = M; p.N = N; p.K = K; p.out = cmat; p.ldo = N; p.status = status;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (status) CU_TRY(cudaMemsetAsync(status, 0, sizeof(int), st));
+    CU_TRY(launch_gemm(out_f32 ? EPI_STORE_F32 : EPI_STORE_BF16, ta, tb, p, sms, st));
+    return VERILLM_OK;
+}
+
+int verillm_op_rmsnorm(const float* x, const void* gain, void* y, int32_t M, int32_t d, float eps, void* cuda_stream) {
+    if (!x || !gain || !y || M < 1 || d < 4) return VERILLM_E_INVAL;
+    if (d % 4 != 0) return VERILLM_E_SHAPE;
+    CU_TRY(launch_rmsnorm(x, gain, y, M, d, eps, reinterpret_cast<cudaStream_t>(cuda_stream)));
+    return VERILLM_OK;
+}
+
+int verillm_op_attention(const void* qkv, const int32_t* cu_seqlens, int32_t batch, int32_t max_seqlen, int32_t M,
+                         int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void* out, void* cuda_stream) {
+    if (!qkv || !cu_seqlens || !out || batch < 1 || max_seqlen < 1 || M < 1) return VERILLM_E_INVAL;
+    if ((head_dim != 64 && head_dim != 128) || n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads != 0)
+        return VERILLM_E_SHAPE;
+    int rc = ensure_init();
+    if (rc) return rc;
+    CU_TRY(launch_attention(qkv, cu_seqlens, batch, max_seqlen, n_heads, n_kv_heads, head_dim, out,
+                            reinterpret_cast<cudaStream_t>(cuda_stream)));
+    return VERILLM_OK;
+}
+
+}  // extern "C"
