@@ -98,6 +98,8 @@ def float_fields(x_rounded: np.ndarray, dtype: str):
 
 @dataclasses.dataclass
 class Model:
+    """`layers` is any sequence of per-layer weight dicts (float64); it may generate them on access."""
+
     n_layers: int
     d_model: int
     n_heads: int
@@ -181,9 +183,8 @@ def silu(z: np.ndarray) -> np.ndarray:
     return z / (1.0 + np.exp(-z))
 
 
-def layer_forward(m: Model, l: int, h: np.ndarray, positions: np.ndarray) -> np.ndarray:
-    """One pre-norm block F_l on a whole sequence h: [T, d_model] -> [T, d_model]."""
-    w = m.layers[l]
+def layer_forward(m: Model, w: Dict[str, np.ndarray], h: np.ndarray, positions: np.ndarray) -> np.ndarray:
+    """One pre-norm block F_l with weights w on a whole sequence h: [T, d_model] -> [T, d_model]."""
     T = h.shape[0]
     a = rmsnorm(h, w["attn_norm"], m.rms_eps)
     q = (a @ w["wq"].T).reshape(T, m.n_heads, m.head_dim)
@@ -197,19 +198,26 @@ def layer_forward(m: Model, l: int, h: np.ndarray, positions: np.ndarray) -> np.
     return u + (silu(f @ w["w_gate"].T) * (f @ w["w_up"].T)) @ w["w_down"].T
 
 
-def forward_prefill(m: Model, tokens: np.ndarray) -> np.ndarray:
-    """All layer-output states of one sequence in a single causal pass (Eq. 1).
+def forward_prefill_batch(m: Model, seqs: Sequence[np.ndarray]) -> List[np.ndarray]:
+    """All layer-output states of every sequence, each in a single causal pass (Eq. 1).
 
-    Returns [n_layers, T, d_model]: entry l is the residual stream after block l+1, i.e. the
-    boundary state S_{l+2} in the paper's numbering, before the final norm."""
-    T = len(tokens)
-    pos = np.arange(T)
-    h = embed_tokens(m, tokens)
-    states = np.empty((m.n_layers, T, m.d_model), dtype=np.float64)
+    Returns one [n_layers, T_b, d_model] array per sequence: entry l is the residual stream after
+    block l+1, i.e. the boundary state S_{l+2} in the paper's numbering, before the final norm.
+    Sequences never interact; the loop runs layer by layer over all of them only so that `m.layers`
+    may be a lazy sequence that materialises one layer's weights at a time."""
+    hs = [embed_tokens(m, np.asarray(t)) for t in seqs]
+    out = [np.empty((m.n_layers, len(t), m.d_model), dtype=np.float64) for t in seqs]
     for l in range(m.n_layers):
-        h = layer_forward(m, l, h, pos)
-        states[l] = h
-    return states
+        w = m.layers[l]
+        for b in range(len(seqs)):
+            hs[b] = layer_forward(m, w, hs[b], np.arange(hs[b].shape[0]))
+            out[b][l] = hs[b]
+    return out
+
+
+def forward_prefill(m: Model, tokens: np.ndarray) -> np.ndarray:
+    """One sequence: [n_layers, T, d_model]."""
+    return forward_prefill_batch(m, [tokens])[0]
 
 
 def forward_decode_kvcache(m: Model, tokens: np.ndarray, precision: str = "f64") -> np.ndarray:
@@ -410,12 +418,15 @@ def verify_prefill(
     committed = as_f64(committed)
     n_check = len(check_seq)
     hidden = np.zeros((m.n_layers, n_check, m.d_model), dtype=np.float64)
+    todo, prefixes = [], []
     for b, toks in enumerate(seqs):
         sel = np.nonzero(np.asarray(check_seq) == b)[0]
         if sel.size == 0:
             continue
         upto = int(np.max(np.asarray(check_pos)[sel])) + 1 if prefix_only else len(toks)
-        states = forward_prefill(m, np.asarray(toks)[:upto])
+        todo.append(sel)
+        prefixes.append(np.asarray(toks)[:upto])
+    for sel, states in zip(todo, forward_prefill_batch(m, prefixes)):
         for slot in sel:
             hidden[:, slot, :] = states[:, int(check_pos[slot]), :]
     stats = compare_stats(hidden, committed, commit_dtype, tol)  # [n_layers, n_check, NSTAT]
