@@ -73,6 +73,7 @@ class Workload:
     check_frac: float
     seed: int
     oracle_weights: str = "bf16"  # "f32": the oracle keeps the fp32 master values
+    token_seed_offset: int = 0  # replicas of one model draw different sequences, checks and tampering
 
     @property
     def seq_len(self) -> int:
@@ -285,7 +286,7 @@ def model_weights(
 def token_streams(wl: Workload) -> np.ndarray:
     """int32 [batch, prompt_len + gen_len] tokens, uniform over the vocabulary."""
     n = wl.n_tokens
-    z = _mix_range(_tensor_key(wl.seed + 1, 0), 0, n, torch.device("cpu"))
+    z = _mix_range(_tensor_key(wl.seed + 1 + wl.token_seed_offset, 0), 0, n, torch.device("cpu"))
     z = torch.bitwise_right_shift(z, 1).bitwise_and_((1 << 62) - 1)
     tok = torch.remainder(z, wl.shape.vocab).to(torch.int32)
     return tok.view(wl.batch, wl.seq_len).numpy().copy()
@@ -300,7 +301,7 @@ def check_positions(wl: Workload, n_check: Optional[int] = None, force: Iterable
     positions (prompt and generated alike), in draw order (unsorted).  `force` pairs are
     placed first (the tampering recipes need their position in the check set)."""
     n = wl.n_check if n_check is None else n_check
-    rng = np.random.Generator(np.random.PCG64(wl.seed + 2))
+    rng = np.random.Generator(np.random.PCG64(wl.seed + 2 + wl.token_seed_offset))
     flat = rng.choice(wl.n_tokens, size=min(n, wl.n_tokens), replace=False)
     forced = [s * wl.seq_len + p for s, p in force]
     if forced:
@@ -313,7 +314,7 @@ def check_positions(wl: Workload, n_check: Optional[int] = None, force: Iterable
 
 
 def tamper_rng(wl: Workload) -> np.random.Generator:
-    return np.random.Generator(np.random.PCG64(wl.seed + 3))
+    return np.random.Generator(np.random.PCG64(wl.seed + 3 + wl.token_seed_offset))
 
 
 def swap_token(tokens: np.ndarray, seq: int, pos: int, vocab: int, rng: np.random.Generator) -> np.ndarray:

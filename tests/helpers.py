@@ -55,3 +55,40 @@ def oracle_tol(**kw) -> vo.Tol:
 def rel_l2(a: np.ndarray, b: np.ndarray) -> np.ndarray:
     """Row-wise ||a-b|| / ||b|| over the last axis."""
     return np.linalg.norm(a - b, axis=-1) / np.maximum(np.linalg.norm(b, axis=-1), 1e-30)
+
+
+class LazyLayers:
+    """Sequence of per-layer float64 weight dicts of a workload, one layer materialised per access.
+    `device` is where the seeded generator runs (the values are identical on any device)."""
+
+    def __init__(self, wl: synth.Workload, n_layers: int, device="cpu"):
+        self.wl, self.n, self.device = wl, n_layers, device
+
+    def __len__(self):
+        return self.n
+
+    def __getitem__(self, l: int):
+        lw = synth.layer_weights(self.wl, l, self.device, torch.bfloat16)
+        return {k: vo.as_f64(bits(v)) for k, v in lw.items()}
+
+
+def oracle_model_streamed(wl: synth.Workload, tokens, device="cpu") -> vo.Model:
+    """Oracle model whose layers are generated on access and whose embedding holds only the rows in use."""
+    s = wl.shape
+    ids = sorted(set(int(t) for t in np.asarray(tokens).reshape(-1)))
+    embed = vo.as_f64(bits(synth.embed_weights(wl, device, torch.bfloat16, rows=torch.tensor(ids))))
+    final = vo.as_f64(bits(synth.final_norm_weights(wl, "cpu", torch.bfloat16)))
+    return vo.Model(s.n_layers, s.d_model, s.n_heads, s.n_kv_heads, s.head_dim, s.d_ffn, s.vocab,
+                    float(s.rope_base), float(s.rms_eps), embed, final, LazyLayers(wl, s.n_layers, device),
+                    {t: i for i, t in enumerate(ids)})
+
+
+def gpu_model(wl: synth.Workload, max_checks: int, device="cuda:0"):
+    """Library handle holding the workload's weights, generated on the device layer by layer."""
+    from paper_2509_24257_b200 import binding as vb
+
+    m = vb.Model(wl.shape, wl.n_tokens, max_checks, wl.batch, device)
+    m.load_globals(synth.embed_weights(wl, device), synth.final_norm_weights(wl, device))
+    for l in range(wl.shape.n_layers):
+        m.load_layer(l, synth.layer_weights(wl, l, device))
+    return m
