@@ -1,0 +1,144 @@
+"""Single steps of the CUDA path against the oracle's pieces, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import verillm_oracle as vo
+from paper_2509_24257_b200 import binding as vb
+from paper_2509_24257_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _rand_bf16(shape, seed, scale=0.5):
+    g = torch.Generator().manual_seed(seed)
+    return (torch.randn(*shape, generator=g) * scale).to(torch.bfloat16)
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 768, 256), (300, 96, 72), (129, 32, 8), (1000, 512, 4096), (2049, 2816, 1024)])
+def test_gemm_matches_textbook_product(M, N, K):
+    # several 128x256 tiles, ragged last row tile, N and K tails
+    a, b = _rand_bf16((M, K), 1), _rand_bf16((N, K), 2)
+    ref = vo.as_f64(H.bits(a)) @ vo.as_f64(H.bits(b)).T
+    c32 = vb.op_gemm(a.to(DEV), b.to(DEV), out_f32=True).cpu().numpy().astype(np.float64)
+    c16 = vb.op_gemm(a.to(DEV), b.to(DEV), out_f32=False).float().cpu().numpy().astype(np.float64)
+    # fp32 accumulation of K products: error ~ sqrt(K) * 2^-24 relative to the row scale
+    assert np.linalg.norm(c32 - ref) <= 2e-5 * np.linalg.norm(ref)
+    assert np.max(H.rel_l2(c32, ref)) <= 5e-5
+    assert np.max(H.rel_l2(c16, ref)) <= 4e-3  # one bf16 rounding of the result
+    assert np.array_equal(c16, vo.round_to_bf16(c32))  # bf16 output = RNE of the fp32 accumulator
+
+
+def test_gemm_rejects_unsupported_shapes():
+    a, b = _rand_bf16((16, 12), 1).to(DEV), _rand_bf16((32, 12), 2).to(DEV)
+    with pytest.raises(vb.VerillmError) as e:
+        vb.op_gemm(a, b)
+    assert e.value.code == vb.E_SHAPE
+
+
+@pytest.mark.parametrize("M,d", [(77, 1024), (5, 4096), (3, 64)])
+def test_rmsnorm_matches_oracle(M, d):
+    g = torch.Generator().manual_seed(3)
+    x = torch.randn(M, d, generator=g) * 3.0
+    gain = (1 + 0.1 * torch.randn(d, generator=g)).to(torch.bfloat16)
+    y = vb.op_rmsnorm(x.to(DEV), gain.to(DEV), 1e-5).float().cpu().numpy().astype(np.float64)
+    ref = vo.rmsnorm(x.numpy().astype(np.float64), vo.as_f64(H.bits(gain)), 1e-5)
+    assert np.max(np.abs(y - ref) / np.maximum(np.abs(ref), 1e-30)) <= 2.0 ** -7  # at most one bf16 step apart
+    assert np.max(H.rel_l2(y, ref)) <= 3e-3
+
+
+@pytest.mark.parametrize("Hq,KV,dh,lens", [
+    (4, 4, 64, [64]), (4, 2, 64, [100, 37, 300, 1]), (8, 2, 128, [129, 64, 515]), (2, 1, 128, [1, 2, 127, 128, 130]),
+])
+def test_attention_matches_oracle(Hq, KV, dh, lens):
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    qkv = _rand_bf16((int(cu[-1]), (Hq + 2 * KV) * dh), 4, 1.0)
+    out = vb.op_attention(qkv.to(DEV), cu, Hq, KV, dh).float().cpu().numpy().astype(np.float64)
+    x = vo.as_f64(H.bits(qkv))
+    for b in range(len(lens)):
+        s, e = int(cu[b]), int(cu[b + 1])
+        q = x[s:e, : Hq * dh].reshape(-1, Hq, dh)
+        k = x[s:e, Hq * dh : (Hq + KV) * dh].reshape(-1, KV, dh)
+        v = x[s:e, (Hq + KV) * dh :].reshape(-1, KV, dh)
+        ref = vo.causal_attention(q, k, v).reshape(e - s, Hq, dh)
+        got = out[s:e].reshape(e - s, Hq, dh)
+        assert np.max(H.rel_l2(got, ref)) <= 1e-2  # bf16 probabilities and output
+        assert np.array_equal(got[0], v[0, [g * KV // Hq for g in range(Hq)]])  # first row = v_0 exactly
+
+
+def _engineered_pairs(d, seed):
+    """Hidden/committed rows that exercise every branch of the comparison."""
+    rng = np.random.default_rng(seed)
+    c = rng.standard_normal(d).astype(np.float32) * 2.0
+    h = (c.astype(np.float64) * (1 + 3e-3 * rng.standard_normal(d))).astype(np.float32)
+    h[0:4] = [1.0 - 2.0 ** -9, 0.5, -1.25, 4e-6]
+    c[0:4] = [1.0, 1.0, 1.25, 0.0]
+    h[4:8] = [0.0, -0.0, 3.0, 1e-41]
+    c[4:8] = [-0.0, 0.0, 3.0, 0.0]
+    return h, c
+
+
+@pytest.mark.parametrize("commit", ["bf16", "f32"])
+def test_compare_same_inputs_counts_are_bit_exact(commit):
+    L, n, d = 3, 37, 1024
+    hs, cs = [], []
+    for i in range(L * n):
+        h, c = _engineered_pairs(d, 100 + i)
+        hs.append(h)
+        cs.append(c)
+    hidden = np.stack(hs).reshape(L, n, d)
+    comm = np.stack(cs).reshape(L, n, d)
+    hidden[1, 5, 17] = np.nan
+    comm[2, 9, 3] = np.inf
+    comm[0, 3] = hidden[0, 3]  # an identical row
+    hidden[2, 11] += 0.5  # a grossly wrong row
+    comm_t = synth.to_commit_dtype(comm.astype(np.float64), commit)
+    comm64 = comm_t.to(torch.float64).numpy()
+    check_seq = (np.arange(n) % 4).astype(np.int32)
+    tol_o = vo.Tol(rel_l2=8e-2, tau_large=0.01, bit_aware=False)
+    tol_g = vb.default_tol(rel_l2=8e-2, tau_large=0.01)
+    rep = vb.compare(torch.from_numpy(hidden).to(DEV), comm_t.to(DEV), check_seq, 4, tol_g).cpu()
+    stats_o = np.transpose(vo.compare_stats(hidden.astype(np.float64), comm64, commit, tol_o), (1, 0, 2))
+    pos_ok, first_bad, seq_ok, score = vo.verdict(stats_o, check_seq, 4, tol_o)
+    for j, nm in enumerate(vo.STAT_NAMES):
+        g, o = rep["stats"][..., j].astype(np.float64), stats_o[..., j]
+        if nm.startswith("n_"):
+            assert np.array_equal(g, o), nm  # integer counts: bit-exact
+        elif nm in ("p_e", "q_small", "z_large", "p_m", "p_w"):
+            assert np.allclose(g, o, rtol=1e-6, atol=0), nm  # ratios of identical integers
+        else:
+            assert np.allclose(g, o, rtol=5e-6, atol=1e-9), nm  # fp32 sums of 1024 terms vs fp64
+    assert np.array_equal(rep["pos_ok"], pos_ok)
+    assert np.array_equal(rep["first_bad_layer"], first_bad)
+    assert np.array_equal(rep["seq_ok"], seq_ok)
+    assert np.allclose(rep["seq_score"], score, rtol=1e-5)
+    assert rep["pos_ok"][3] == 1 and rep["pos_ok"][5] == 0 and rep["pos_ok"][9] == 0 and rep["pos_ok"][11] == 0
+
+
+def test_bit_aware_verdict_matches_oracle_on_same_inputs():
+    L, n, d = 2, 16, 512
+    rng = np.random.default_rng(7)
+    comm = rng.standard_normal((L, n, d)).astype(np.float32)
+    hidden = comm.copy()
+    # rows 0..7: honest-like (tiny relative noise); rows 8..15: heavy noise that scrambles exponents
+    hidden[:, :8] *= (1 + 1e-4 * rng.standard_normal((L, 8, d))).astype(np.float32)
+    hidden[:, 8:] *= (1 + 0.4 * rng.standard_normal((L, 8, d))).astype(np.float32)
+    comm_t = synth.to_commit_dtype(comm.astype(np.float64), "f32")
+    kw = dict(rel_l2=0.0, bit_aware=True, pw_min=0.5, pm_min=-1.0, e_w=1e-3)
+    rep = vb.compare(torch.from_numpy(hidden).to(DEV), comm_t.to(DEV), np.zeros(n, np.int32), 1, vb.default_tol(**kw)).cpu()
+    tol_o = vo.Tol(**kw)
+    stats_o = np.transpose(vo.compare_stats(hidden.astype(np.float64), comm.astype(np.float64), "f32", tol_o), (1, 0, 2))
+    pos_ok, first_bad, _, _ = vo.verdict(stats_o, np.zeros(n, np.int32), 1, tol_o)
+    assert np.array_equal(rep["pos_ok"], pos_ok) and np.array_equal(rep["first_bad_layer"], first_bad)
+    assert pos_ok[:8].all() and not pos_ok[8:].any()
+
+
+def test_seeded_generator_is_identical_on_device():
+    wl = synth.WORKLOADS["small"]
+    cpu = synth.layer_weights(wl, 1, "cpu")
+    gpu = synth.layer_weights(wl, 1, DEV)
+    assert all(torch.equal(cpu[k], gpu[k].cpu()) for k in cpu)
+    rows = torch.tensor([0, 31999, 17])
+    assert torch.equal(synth.embed_weights(wl, DEV, rows=rows).cpu(), synth.embed_weights(wl, "cpu")[rows])

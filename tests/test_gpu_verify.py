@@ -1,0 +1,252 @@
+"""End-to-end parity of the verifier path (C ABI on a B200) against the CPU oracle on the same seeded inputs.
+
+Bars: recomputed hidden states within relative L2 <= 2e-2 per checked position and layer; verdicts,
+first failing layers and indices identical for every cell outside the gray band (oracle rel-L2 <= tol/2
+or >= 2 tol; the traces are built so that no intended cell lies inside it); integer work bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import verillm_oracle as vo
+from paper_2509_24257_b200 import binding as vb
+from paper_2509_24257_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+HIDDEN_TOL = 2e-2
+TOL = 5e-2
+REL = vo.STAT_NAMES.index("rel_l2")
+
+
+def run_both(model, om, wl, tokens, committed64, check_seq, check_pos, commit="bf16", prefix_only=False,
+             tol_kw=None, seqs=None, cu=None):
+    """Feeds the same tokens / committed states / check set to the CUDA path and to the oracle."""
+    tol_kw = tol_kw or {}
+    comm_t = synth.to_commit_dtype(committed64, commit)
+    seqs = list(tokens) if seqs is None else seqs
+    cu = synth.cu_seqlens(wl) if cu is None else cu
+    flat = torch.from_numpy(np.concatenate([np.asarray(s) for s in seqs]).astype(np.int32)).to(DEV)
+    rep = model.verify_prefill(flat, cu, comm_t.to(DEV), check_seq, check_pos, vb.default_tol(**tol_kw), want_hidden=True)
+    torch.cuda.synchronize()
+    g = rep.cpu()
+    o = vo.verify_prefill(om, seqs, comm_t.to(torch.float64).numpy(), check_seq, check_pos, vo.Tol(**tol_kw), commit,
+                          prefix_only=prefix_only)
+    return g, o
+
+
+def assert_parity(g, o, tol=TOL, expect_reject=(), expect_gray=()):
+    assert g["status"] == 0
+    # hidden states: the first gate
+    rel = H.rel_l2(g["hidden"], o.hidden)
+    assert rel.max() <= HIDDEN_TOL, f"hidden-state rel-L2 {rel.max():.3e}"
+    # verdicts: identical wherever the oracle's cell is outside the gray band
+    o_rel = o.stats[..., REL]  # [n_check, n_layers]
+    gray = (o_rel > tol / 2) & (o_rel < 2 * tol)
+    gray_pos = gray.any(axis=1)
+    for s in np.nonzero(gray_pos)[0]:
+        assert s in expect_gray, f"slot {s} unexpectedly inside the gray band ({o_rel[s].max():.3e})"
+    clear = ~gray_pos
+    assert np.array_equal(g["pos_ok"][clear], o.pos_ok[clear])
+    assert np.array_equal(g["first_bad_layer"][clear], o.first_bad_layer[clear])
+    for s in expect_reject:
+        assert o.pos_ok[s] == 0 and g["pos_ok"][s] == 0
+    if not gray_pos.any():
+        assert np.array_equal(g["seq_ok"], o.seq_ok)
+        # |MAE_gpu - MAE_oracle| <= mean|h_gpu - h_oracle| <= rms(h_gpu - h_oracle) <= 2e-2 rms(h)
+        bound = HIDDEN_TOL * float(np.sqrt(np.mean(o.hidden ** 2))) * 1.5 + 1e-7
+        assert np.all(np.abs(g["seq_score"] - o.seq_score) <= bound)
+    # statistics: same quantity computed from states that differ by <= 2e-2 of the state norm
+    g_rel = g["stats"][..., REL]
+    assert np.all(np.abs(g_rel - o_rel) <= HIDDEN_TOL * 1.2 + 1e-6)
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    wl = synth.WORKLOADS["tiny"]
+    tokens = synth.token_streams(wl)
+    om = H.oracle_model(wl)
+    cs, cp = synth.check_positions(wl)  # all 64 positions, in draw order
+    committed = H.oracle_committed(om, tokens, cs, cp, "bf16")
+    model = H.gpu_model(wl, len(cs))
+    yield wl, tokens, om, cs, cp, committed, model
+    model.close()
+
+
+def test_tiny_honest_trace_accepts_everywhere(tiny):
+    wl, tokens, om, cs, cp, committed, model = tiny
+    assert len(cs) == 64 and sorted(cp.tolist()) == list(range(64))
+    g, o = run_both(model, om, wl, tokens, committed, cs, cp)
+    assert_parity(g, o)
+    assert g["pos_ok"].all() and g["seq_ok"].tolist() == [1]
+    assert model.last_launch_count() == 3 + 7 * wl.shape.n_layers + 2
+
+
+def test_tiny_noise_at_three_positions_is_rejected_exactly_there(tiny):
+    wl, tokens, om, cs, cp, committed, model = tiny
+    rng = synth.tamper_rng(wl)
+    bad = sorted(rng.choice(len(cs), size=3, replace=False).tolist())
+    tampered = synth.add_state_noise(committed, bad, None, 0.5, rng)  # 0.5 x RMS = 10 x tol
+    g, o = run_both(model, om, wl, tokens, tampered, cs, cp)
+    assert_parity(g, o, expect_reject=bad)
+    assert sorted(np.nonzero(g["pos_ok"] == 0)[0].tolist()) == bad
+    assert g["seq_ok"].tolist() == [0] and (g["first_bad_layer"][bad] == 0).all()
+
+
+def test_tiny_f32_trace_and_bit_aware_statistics(tiny):
+    wl, tokens, om, cs, cp, committed, model = tiny
+    g, o = run_both(model, om, wl, tokens, committed, cs, cp, commit="f32", tol_kw=dict(tau_large=0.05))
+    assert_parity(g, o)
+    # the counts are integers of d_model elements and partition it
+    st = g["stats"]
+    n_mis = st[..., vo.STAT_NAMES.index("n_exp_mismatch")]
+    assert np.all(n_mis == np.round(n_mis)) and np.all(n_mis <= wl.shape.d_model)
+    assert np.allclose(st[..., vo.STAT_NAMES.index("p_e")], n_mis / wl.shape.d_model)
+    # honest noise: few exponent mismatches on either side
+    assert st[..., vo.STAT_NAMES.index("p_e")].mean() < 0.05 and o.stats[..., vo.STAT_NAMES.index("p_e")].mean() < 0.05
+
+
+def test_tiny_results_are_deterministic(tiny):
+    wl, tokens, om, cs, cp, committed, model = tiny
+    comm = synth.to_commit_dtype(committed, "bf16").to(DEV)
+    flat = torch.from_numpy(tokens.reshape(-1)).to(DEV)
+    a = model.verify_prefill(flat, synth.cu_seqlens(wl), comm, cs, cp, want_hidden=True).cpu()
+    b = model.verify_prefill(flat, synth.cu_seqlens(wl), comm, cs, cp, want_hidden=True).cpu()
+    assert np.array_equal(a["stats"], b["stats"]) and np.array_equal(a["hidden"], b["hidden"])
+
+
+def test_ragged_batch_duplicates_and_order(tiny):
+    """Sequences of different lengths (one of length 1), duplicate and unsorted check positions."""
+    wl, tokens, om, _, _, _, _ = tiny
+    rng = np.random.default_rng(5)
+    lens = [57, 1, 130, 64]
+    seqs = [rng.integers(0, wl.shape.vocab, n).astype(np.int32) for n in lens]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    cs = np.array([2, 0, 2, 1, 3, 2, 0, 2], dtype=np.int32)
+    cp = np.array([129, 0, 5, 0, 63, 129, 56, 77], dtype=np.int32)  # slot 0 and 5 name the same position
+    committed = np.zeros((wl.shape.n_layers, len(cs), wl.shape.d_model))
+    for i, (s, p) in enumerate(zip(cs, cp)):
+        committed[:, i] = vo.forward_decode_kvcache(om, seqs[s][: p + 1], "bf16")[:, p]
+    committed = synth.add_state_noise(committed, [5], None, 0.5, rng)  # tamper one of the two duplicates
+    model = vb.Model(wl.shape, int(cu[-1]), len(cs), len(lens), DEV)
+    model.load_globals(synth.embed_weights(wl, DEV), synth.final_norm_weights(wl, DEV))
+    model.load_layer(0, synth.layer_weights(wl, 0, DEV))
+    g, o = run_both(model, om, wl, None, committed, cs, cp, commit="f32", seqs=seqs, cu=cu)
+    assert_parity(g, o, expect_reject=[5])
+    assert g["pos_ok"].tolist() == [1, 1, 1, 1, 1, 0, 1, 1]
+    assert g["seq_ok"].tolist() == [1, 1, 0, 1]
+    assert np.array_equal(g["hidden"][:, 0], g["hidden"][:, 5])  # same position gathered twice, bit-identical
+    # no checks at all: every sequence accepted with score 0
+    flat = torch.from_numpy(np.concatenate(seqs)).to(DEV)
+    rep = model.verify_prefill(flat, cu, None, [], []).cpu()
+    assert rep["seq_ok"].tolist() == [1, 1, 1, 1] and rep["seq_score"].tolist() == [0, 0, 0, 0]
+    model.close()
+
+
+def test_argument_errors_launch_nothing(tiny):
+    wl, tokens, om, cs, cp, committed, model = tiny
+    comm = synth.to_commit_dtype(committed, "bf16").to(DEV)
+    flat = torch.from_numpy(tokens.reshape(-1)).to(DEV)
+    cu = synth.cu_seqlens(wl)
+
+    def code(**kw):
+        args = dict(tokens=flat, cu_seqlens=cu, committed=comm, check_seq=cs, check_pos=cp)
+        args.update(kw)
+        with pytest.raises(vb.VerillmError) as e:
+            model.verify_prefill(**args)
+        return e.value.code
+
+    bad_pos = cp.copy(); bad_pos[3] = 64
+    assert code(check_pos=bad_pos) == vb.E_RANGE
+    bad_seq = cs.copy(); bad_seq[0] = 1
+    assert code(check_seq=bad_seq) == vb.E_RANGE
+    assert code(cu_seqlens=[0, 65]) == vb.E_SHAPE  # more tokens than the handle was sized for
+    assert code(cu_seqlens=[0, 40, 30]) in (vb.E_RANGE, vb.E_SHAPE)
+    assert code(cu_seqlens=[1, 64]) == vb.E_RANGE
+    with pytest.raises(vb.VerillmError) as e:
+        vb.Model(synth.ModelShape(1, 256, 4, 4, 96, 768, 1024), 64, 4, 1, DEV)  # head_dim 96
+    assert e.value.code == vb.E_SHAPE
+    # a token id outside the vocabulary is clamped on the device, flagged, and rejects everything
+    bad_tok = flat.clone(); bad_tok[10] = wl.shape.vocab + 5
+    rep = model.verify_prefill(bad_tok, cu, comm, cs, cp).cpu()
+    assert rep["status"] == vb.DEV_TOKEN_RANGE and not rep["pos_ok"].any() and rep["seq_ok"].tolist() == [0]
+    # and the handle keeps working afterwards
+    assert model.verify_prefill(flat, cu, comm, cs, cp).cpu()["pos_ok"].all()
+
+
+@pytest.fixture(scope="module")
+def small():
+    wl = synth.WORKLOADS["small"]
+    tokens = synth.token_streams(wl)
+    om = H.oracle_model(wl)
+    rng = synth.tamper_rng(wl)
+    # the token-swap position is forced into the check set (its later positions move only slightly)
+    swap_seq, swap_pos = 1, wl.prompt_len + int(rng.integers(0, wl.gen_len))
+    cs, cp = synth.check_positions(wl, force=[(swap_seq, swap_pos)])
+    committed = H.oracle_committed(om, tokens, cs, cp, "bf16")
+    model = H.gpu_model(wl, len(cs))
+    yield wl, tokens, om, cs, cp, committed, model, rng, (swap_seq, swap_pos)
+    model.close()
+
+
+def test_small_honest_trace(small):
+    wl, tokens, om, cs, cp, committed, model, rng, _ = small
+    assert len(cs) == 20
+    g, o = run_both(model, om, wl, tokens, committed, cs, cp, prefix_only=True)
+    assert_parity(g, o)
+    assert g["pos_ok"].all() and g["seq_ok"].all()
+
+
+def test_small_substituted_token_is_caught_at_its_position(small):
+    wl, tokens, om, cs, cp, committed, model, rng, (sq, sp) = small
+    forged = synth.swap_token(tokens, sq, sp, wl.shape.vocab, rng)
+    later = [i for i in range(len(cs)) if cs[i] == sq and cp[i] > sp]  # may drift into the gray band
+    g, o = run_both(model, om, wl, forged, committed, cs, cp, prefix_only=True)
+    assert_parity(g, o, expect_reject=[0], expect_gray=later)
+    assert g["seq_ok"][sq] == 0 and o.seq_ok[sq] == 0
+    others = [b for b in range(wl.batch) if b != sq]
+    assert g["seq_ok"][others].all() and o.seq_ok[others].all()
+
+
+def test_small_layer_output_perturbation_of_ten_times_tolerance(small):
+    wl, tokens, om, cs, cp, committed, model, rng, _ = small
+    slot, layer = 7, 2
+    tampered = synth.add_state_noise(committed, [slot], [layer], 10 * TOL, rng)
+    g, o = run_both(model, om, wl, tokens, tampered, cs, cp, prefix_only=True)
+    assert_parity(g, o, expect_reject=[slot])
+    assert g["first_bad_layer"][slot] == layer and (np.delete(g["pos_ok"], slot) == 1).all()
+
+
+def test_decode_commit_matches_oracle_decode_and_verifies_as_honest(small):
+    wl, tokens, om, cs, cp, committed, model, rng, _ = small
+    ref = H.oracle_committed(om, tokens, cs, cp, "f64")
+    flat = torch.from_numpy(tokens.reshape(-1)).to(DEV)
+    for n_prefill in (wl.prompt_len, 0, 300):
+        trace = model.decode_commit(flat, synth.cu_seqlens(wl), n_prefill, cs, cp, torch.float32)
+        rel = H.rel_l2(trace.double().cpu().numpy(), ref)
+        assert rel.max() <= HIDDEN_TOL, (n_prefill, rel.max())
+    trace = model.decode_commit(flat, synth.cu_seqlens(wl), wl.prompt_len, cs, cp, torch.bfloat16)
+    rep = model.verify_prefill(flat, synth.cu_seqlens(wl), trace.contiguous(), cs, cp).cpu()
+    assert rep["status"] == 0 and rep["pos_ok"].all() and rep["seq_ok"].all()
+    assert 0 < rep["stats"][..., REL].max() <= TOL / 2  # decode and prefill differ, but only by rounding noise
+
+
+def test_llama8b_width_reduced_depth():
+    """Full layer widths (d 4096, 32/8 heads of 128, FFN 14336), two layers, ragged check set."""
+    wl = synth.WORKLOADS["llama8b"].with_layers(2).with_batch(3, 200, 184)
+    tokens = synth.token_streams(wl)
+    cs = np.array([0, 0, 1, 2, 2, 1], dtype=np.int32)
+    cp = np.array([0, 95, 130, 17, 127, 64], dtype=np.int32)
+    om = H.oracle_model_streamed(wl, tokens, DEV)
+    model = H.gpu_model(wl, len(cs))
+    pre = vo.verify_prefill(om, list(tokens), np.zeros((2, len(cs), wl.shape.d_model)), cs, cp, vo.Tol(), "bf16",
+                            prefix_only=True)
+    honest = vo.round_to_bf16(pre.hidden)  # a prover that ran the same pass and serialised to bf16
+    rng = synth.tamper_rng(wl)
+    tampered = synth.add_state_noise(honest, [3], [1], 10 * TOL, rng)
+    g, o = run_both(model, om, wl, tokens, tampered, cs, cp, prefix_only=True)
+    assert_parity(g, o, expect_reject=[3])
+    assert g["pos_ok"].tolist() == [1, 1, 1, 0, 1, 1] and g["seq_ok"].tolist() == [1, 1, 0]
+    assert g["first_bad_layer"][3] == 1
+    model.close()
