@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the verifier prefill: verified tokens/s at the Llama-3-8B shape on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload llama8b]
+
+A step is one verillm_verify_prefill call over one synthetic batch (8 sequences of 512 prompt + 512
+generated tokens, 1 % of positions checked at every layer, 10 % of sequences tampered): embedding,
+32 transformer blocks with the fused gather-and-compare epilogue, verdict.  Weights (15 GB) are
+re-streamed from HBM every step, far more than the 126 MB L2, so no flush is needed between steps.
+With N > 1 (torchrun) every rank runs an independent replica on its own sequences; there is no
+collective on the data path.  Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC, UNIT = "verified_tokens_per_sec", "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+TOL_REL_L2 = 5e-2
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index, self.proc, self.lines = gpu_index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100", "-i",
+                 str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ts, line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7 or not (t0 <= ts <= t1 + 0.2):
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------- CPU arm
+
+
+def oracle_sample(wl, budget_s: float, device_for_weights: str):
+    """Builds a bounded sample of the workload for the CPU oracle: one sequence prefix and the first
+    layers, sized from a short calibration run so that one pass costs about `budget_s` seconds.
+    Returns (run, description) where run() executes one pass and returns (tokens, seconds, layers)."""
+    import torch
+    from oracle import verillm_oracle as vo
+    from paper_2509_24257_b200 import synth
+
+    def bits(t):
+        return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+    shape = wl.shape
+    tokens = synth.token_streams(wl)[0]
+    ids = sorted(set(int(t) for t in tokens))
+    embed = vo.as_f64(bits(synth.embed_weights(wl, device_for_weights, rows=torch.tensor(ids))))
+    rows = {t: i for i, t in enumerate(ids)}
+    final = vo.as_f64(bits(synth.final_norm_weights(wl, "cpu")))
+    layer0 = {k: vo.as_f64(bits(v)) for k, v in synth.layer_weights(wl, 0, device_for_weights).items()}
+
+    def model(n_layers):
+        return vo.Model(n_layers, shape.d_model, shape.n_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn,
+                        shape.vocab, float(shape.rope_base), float(shape.rms_eps), embed, final,
+                        [layer0] * n_layers, rows)
+
+    # calibration: one layer on 64 tokens (the cost is close to linear in tokens x layers)
+    t0 = time.perf_counter()
+    vo.forward_prefill_batch(model(1), [tokens[:64]])
+    per_token_layer = (time.perf_counter() - t0) / 64.0
+    n_layers = 2 if shape.n_layers >= 2 else 1
+    T = int(min(len(tokens), max(64, (budget_s / (per_token_layer * n_layers)) // 64 * 64)))
+    om = model(n_layers)
+    n_chk = max(1, int(round(wl.check_frac * T)))
+    check_pos = np.linspace(0, T - 1, n_chk).astype(np.int32)
+    check_seq = np.zeros(n_chk, dtype=np.int32)
+    committed = np.zeros((n_layers, n_chk, shape.d_model))
+    tol = vo.Tol(rel_l2=TOL_REL_L2)
+
+    def run():
+        t0 = time.perf_counter()
+        vo.verify_prefill(om, [tokens[:T]], committed, check_seq, check_pos, tol, "bf16")
+        return T, time.perf_counter() - t0, n_layers
+
+    desc = (f"oracle (numpy fp64) on 1 sequence x {T} tokens x {n_layers} of {shape.n_layers} layers at full width, "
+            f"{n_chk} checked positions; tokens/s scaled by {n_layers}/{shape.n_layers} to the full depth")
+    return run, desc
+
+
+def cpu_cores() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+    except Exception:
+        n = 1
+    return int(min(n, len(os.sched_getaffinity(0))))
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", 0))
+    if rank != 0:
+        return
+    import torch
+
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    budget = max(1.0, min(20.0, 150.0 / (args.steps + args.warmup)))
+    run, desc = oracle_sample(wl, budget, dev)
+    for _ in range(args.warmup):
+        run()
+    tot_tokens, tot_s = 0.0, 0.0
+    for _ in range(args.steps):
+        T, s, nl = run()
+        tot_tokens += T * nl / wl.shape.n_layers
+        tot_s += s
+    value = tot_tokens / tot_s
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * tot_s / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "timing": "host wall clock; the oracle runs on the host cores"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------- GPU arm
+
+
+def build_job(wl, device):
+    """Model handle plus one batch of inputs resident on the device (weights generated in place)."""
+    import torch
+    from paper_2509_24257_b200 import binding as vb, synth
+
+    cs, cp = synth.check_positions(wl)
+    model = vb.Model(wl.shape, wl.n_tokens, len(cs), wl.batch, device)
+    model.load_globals(synth.embed_weights(wl, device), synth.final_norm_weights(wl, device))
+    for l in range(wl.shape.n_layers):
+        model.load_layer(l, synth.layer_weights(wl, l, device))
+    torch.cuda.empty_cache()
+    tokens = synth.token_streams(wl)
+    cu = synth.cu_seqlens(wl)
+    flat = torch.from_numpy(tokens.reshape(-1)).to(device)
+    # the prover's trace: teacher-forced bf16 KV-cache decode after a parallel pass over the prompts
+    t0 = time.perf_counter()
+    committed = model.decode_commit(flat, cu, wl.prompt_len, cs, cp, torch.bfloat16).contiguous()
+    trace_s = time.perf_counter() - t0
+    # tamper ceil(10 %) of the sequences, alternating a substituted token and state noise of 10 x tol
+    rng = synth.tamper_rng(wl)
+    n_bad = int(math.ceil(0.1 * wl.batch))
+    bad_seqs = sorted(rng.choice(wl.batch, size=n_bad, replace=False).tolist())
+    tampered_tokens = tokens
+    comm_host = committed.float().cpu().numpy().astype(np.float64)
+    for i, b in enumerate(bad_seqs):
+        slots = np.nonzero(cs == b)[0]
+        if slots.size == 0:
+            continue
+        slot = int(slots[0])
+        if i % 2 == 0:
+            tampered_tokens = synth.swap_token(tampered_tokens, b, int(cp[slot]), wl.shape.vocab, rng)
+        else:
+            comm_host = synth.add_state_noise(comm_host, [slot], [int(rng.integers(0, wl.shape.n_layers))],
+                                              10 * TOL_REL_L2, rng)
+    committed = synth.to_commit_dtype(comm_host, "bf16").to(device)
+    flat = torch.from_numpy(tampered_tokens.reshape(-1)).to(device)
+    return model, flat, tampered_tokens, cu, cs, cp, committed, bad_seqs, trace_s
+
+
+def run_ours(args, wl):
+    import torch
+    from paper_2509_24257_b200 import binding as vb, dist as vdist
+
+    rank, world, local = vdist.init()
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    wl_r = vdist.replica_workload(wl, rank)
+    model, flat, tokens_host, cu, cs, cp, committed, bad_seqs, trace_s = build_job(wl_r, device)
+    tol = vb.default_tol(rel_l2=TOL_REL_L2)
+    report = vb.Report(len(cs), wl.shape.n_layers, wl.batch, wl.shape.d_model, device, False)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        model.verify_prefill(flat, cu, committed, cs, cp, tol, report=report, stream=stream)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    # ---- device-resident timing: exactly K steps between two events
+    sampler = ClockSampler(int(os.environ.get("CUDA_VISIBLE_DEVICES", "0").split(",")[local]) if
+                           os.environ.get("CUDA_VISIBLE_DEVICES") else local)
+    sampler.start()
+    time.sleep(0.3)
+    vdist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    vdist.barrier()
+    seconds = e0.elapsed_time(e1) / 1e3
+    clocks = sampler.stop(t_wall0, t_wall1)
+    res = report.cpu()
+    launches = model.last_launch_count() * args.steps
+    value = vdist.aggregate_throughput(float(wl.n_tokens * args.steps), seconds)
+    slowest = vdist.max_over_ranks(seconds)
+
+    # ---- end to end: host buffers in, report out, every step
+    pin = lambda t: t.cpu().pin_memory()
+    tok_pin, comm_pin = pin(flat), pin(committed)
+    out_pin = {k: torch.empty_like(getattr(report, k), device="cpu").pin_memory()
+               for k in ("stats", "pos_ok", "first_bad_layer", "seq_ok", "seq_score", "status")}
+    tok_dev, comm_dev = torch.empty_like(flat), torch.empty_like(committed)
+
+    def e2e_step():
+        tok_dev.copy_(tok_pin, non_blocking=True)
+        comm_dev.copy_(comm_pin, non_blocking=True)
+        model.verify_prefill(tok_dev, cu, comm_dev, cs, cp, tol, report=report, stream=stream)
+        for k, buf in out_pin.items():
+            buf.copy_(getattr(report, k), non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_step()
+    vdist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()
+    e2e_seconds = time.perf_counter() - t0
+    vdist.barrier()
+    e2e_value = vdist.aggregate_throughput(float(wl.n_tokens * args.steps), e2e_seconds)
+    h2d = tok_pin.numel() * 4 + comm_pin.numel() * comm_pin.element_size() + 4 * (len(cu) + 2 * len(cs))
+    d2h = sum(b.numel() * b.element_size() for b in out_pin.values())
+
+    # ---- per-kernel times (second pass with one event per launch) for the roofline of the dominant kernel
+    peaks, peaks_kind = measured_peaks()
+    model.profile_enable(True)
+    acc = {}
+    for _ in range(min(args.steps, 5)):
+        step()
+        for k, (ms, n) in model.profile_read().items():
+            a = acc.setdefault(k, [0.0, 0])
+            a[0] += ms
+            a[1] += n
+    model.profile_enable(False)
+    s = wl.shape
+    M = wl.n_tokens
+    flops_per_launch = {
+        "gemm_qkv_rope": 2.0 * M * (s.d_q + 2 * s.d_kv) * s.d_model,
+        "gemm_o_resid": 2.0 * M * s.d_model * s.d_q,
+        "gemm_gate_up_swiglu": 2.0 * M * 2 * s.d_ffn * s.d_model,
+        "gemm_down_resid_compare": 2.0 * M * s.d_model * s.d_ffn,
+        "attention": 4.0 * s.n_heads * s.head_dim * M * (wl.seq_len + 1) / 2.0,
+    }
+    kernels = {}
+    for k, (ms, n) in acc.items():
+        if n == 0:
+            continue
+        per = ms / n
+        kernels[k] = {"launches_per_step": n // min(args.steps, 5), "ms_per_launch": round(per, 4)}
+        if k in flops_per_launch:
+            kernels[k]["tflops"] = round(flops_per_launch[k] / (per * 1e-3) / 1e12, 1)
+    dom = "gemm_gate_up_swiglu"
+    achieved = flops_per_launch[dom] / (acc[dom][0] / acc[dom][1] * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "TFLOP/s",
+                "frac": round(achieved / peak, 4), "traffic": None,
+                "peak_kind": f"bf16 sustained, of {peaks_kind}", "kernels": kernels}
+
+    if rank == 0:
+        run, desc = oracle_sample(wl, 12.0, str(device)) if args.gpus == 1 else (None, None)
+        cpu_baseline = None
+        if run is not None:
+            T, sec, nl = run()
+            cpu_baseline = {"value": T * nl / wl.shape.n_layers / sec, "unit": UNIT, "cores": cpu_cores(),
+                            "kind": "oracle", "sample": desc}
+        total_tflops = wl.total_flops() * args.gpus * args.steps / slowest / 1e12
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * slowest / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {
+                "workload": wl.name, "batch": wl.batch, "seq_len": wl.seq_len, "n_check": int(len(cs)),
+                "tampered_sequences": bad_seqs, "parallelism": f"replicas x{args.gpus}",
+                "l2": "inputs larger than L2 (15 GB of weights streamed per step)",
+                "trace": f"committed states from verillm_decode_commit ({trace_s:.1f} s, untimed)",
+            },
+            "model_tflops": round(total_tflops, 1),
+            "pct_of_bf16_peak": {"of_measured_burst": round(total_tflops / args.gpus / peaks["bf16_tflops"], 4),
+                                 "of_measured_sustained": round(total_tflops / args.gpus / peaks["bf16_tflops_sustained"], 4),
+                                 "of_nominal_2250": round(total_tflops / args.gpus / 2250.0, 4), "peaks": peaks_kind},
+            "verdicts": {"seq_ok": res["seq_ok"].tolist(), "positions_rejected": int((res["pos_ok"] == 0).sum()),
+                         "status": res["status"]},
+            "clocks": clocks, "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                                     "d2h_bytes_per_step": int(d2h)},
+            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line))
+    model.close()
+    vdist.shutdown()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    from paper_2509_24257_b200 import synth
+
+    wl = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

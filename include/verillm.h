@@ -194,6 +194,25 @@ int verillm_op_rmsnorm(const float *x, const void *gain, void *y, int32_t m, int
 int verillm_op_attention(const void *qkv, const int32_t *cu_seqlens, int32_t batch, int32_t max_seqlen, int32_t m,
                          int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void *out, void *cuda_stream);
 
+/* Per-kernel timing of verify_prefill, for the roofline report (measurement aid, not part of the method).
+ * While enabled, every verify_prefill call records one CUDA event after each launch on the caller's
+ * stream; verillm_profile_read waits for the last call and returns, per class below, the summed
+ * milliseconds and the number of launches (HOST arrays of VERILLM_PROF_NCLASS entries).  Enabling creates
+ * the events once (not on the hot path); the events add a few microseconds per launch. */
+enum {
+    VERILLM_PROF_SETUP = 0,       /* index maps, slot lists, embedding gather */
+    VERILLM_PROF_RMSNORM = 1,
+    VERILLM_PROF_GEMM_QKV = 2,    /* + rotary epilogue */
+    VERILLM_PROF_ATTENTION = 3,
+    VERILLM_PROF_GEMM_O = 4,      /* + residual */
+    VERILLM_PROF_GEMM_GATE_UP = 5,/* + SwiGLU */
+    VERILLM_PROF_GEMM_DOWN = 6,   /* + residual + gather-and-compare */
+    VERILLM_PROF_VERDICT = 7,
+    VERILLM_PROF_NCLASS = 8
+};
+int verillm_profile_enable(verillm_model *model, int32_t on);
+int verillm_profile_read(verillm_model *model, float *ms, int32_t *launches);
+
 void verillm_free(verillm_model *model);
 const char *verillm_strerror(int code);
 /* Number of kernel launches the last verify_prefill call on this handle enqueued. */

@@ -63,7 +63,7 @@ def round_to_bf16(x: np.ndarray) -> np.ndarray:
         _, e = np.frexp(xf)
         q = np.ldexp(1.0, np.maximum(e - 8, -133))
         r = np.rint(xf / q) * q
-        r = np.where(np.abs(r) >= np.ldexp(1.0, 128), np.sign(r) * np.inf, r)
+        r = np.where(np.abs(r) >= np.ldexp(1.0, 128), np.copysign(np.inf, r), r)
         out[fin] = r
     return out
 

@@ -29,8 +29,10 @@ EXPORTS = (
     "verillm_default_tol", "verillm_load_weights", "verillm_load_layer", "verillm_load_globals",
     "verillm_verify_prefill", "verillm_decode_commit", "verillm_compare", "verillm_op_gemm",
     "verillm_op_rmsnorm", "verillm_op_attention", "verillm_free", "verillm_strerror",
-    "verillm_last_launch_count",
+    "verillm_last_launch_count", "verillm_profile_enable", "verillm_profile_read",
 )
+PROF_CLASSES = ("setup", "rmsnorm", "gemm_qkv_rope", "attention", "gemm_o_resid", "gemm_gate_up_swiglu",
+                "gemm_down_resid_compare", "verdict")
 
 
 class VerillmError(RuntimeError):
@@ -107,6 +109,10 @@ def lib() -> C.CDLL:
         L.verillm_op_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.verillm_op_rmsnorm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p]
         L.verillm_op_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.verillm_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+        L.verillm_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+        L.verillm_profile_enable.restype = C.c_int
+        L.verillm_profile_read.restype = C.c_int
         for name in ("verillm_load_weights", "verillm_load_layer", "verillm_load_globals", "verillm_verify_prefill",
                      "verillm_decode_commit", "verillm_compare", "verillm_op_gemm", "verillm_op_rmsnorm",
                      "verillm_op_attention"):
@@ -265,6 +271,18 @@ class Model:
         if int(status.item()) != 0:
             raise RuntimeError(f"verillm_decode_commit: device status {int(status.item())}")
         return out[:, :n_check]
+
+    def profile_enable(self, on: bool = True) -> None:
+        with torch.cuda.device(self.device):
+            _check(lib().verillm_profile_enable(self._h, int(on)), "verillm_profile_enable")
+
+    def profile_read(self) -> Dict[str, tuple]:
+        """{kernel class: (milliseconds, launches)} of the last verify_prefill call."""
+        ms = (C.c_float * len(PROF_CLASSES))()
+        n = (C.c_int32 * len(PROF_CLASSES))()
+        with torch.cuda.device(self.device):
+            _check(lib().verillm_profile_read(self._h, ms, n), "verillm_profile_read")
+        return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(PROF_CLASSES)}
 
     def last_launch_count(self) -> int:
         return int(lib().verillm_last_launch_count(self._h))

@@ -44,6 +44,14 @@ struct DecodeState {
     int* ints = nullptr;  // index scratch: 6 * max_tokens + 3 * max_checks
 };
 
+// Optional per-kernel timing: one event after every launch of a verify_prefill call.
+struct Profile {
+    bool on = false;
+    std::vector<cudaEvent_t> ev;
+    std::vector<int> cls;
+    int n = 0;
+};
+
 }  // namespace
 
 struct verillm_model {
@@ -61,10 +69,19 @@ struct verillm_model {
     float2* rope_cs = nullptr;
     CUtensorMap t_xn, t_attn, t_mid;
     DecodeState dec;
+    Profile prof;
     int last_launches = 0;
 };
 
 namespace {
+
+inline void prof_mark(verillm_model* m, int cls, cudaStream_t st) {
+    Profile& p = m->prof;
+    if (!p.on || p.n >= static_cast<int>(p.ev.size())) return;
+    cudaEventRecord(p.ev[p.n], st);
+    p.cls[p.n] = cls;
+    ++p.n;
+}
 
 int ensure_init() {
     static bool done[64] = {false};
@@ -175,15 +192,21 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
     p.M = r.M;
 
     CU_TRY(launch_rmsnorm(m->resid, w.attn_norm, m->xn, r.M, c.d_model, c.rms_eps, st));
+    prof_mark(m, VERILLM_PROF_RMSNORM, st);
     p.N = m->n_qkv; p.K = c.d_model; p.out = m->qkv; p.ldo = m->n_qkv;
     p.rope_cs = m->rope_cs; p.pos_of_token = m->pos_of_token; p.head_dim = c.head_dim; p.rope_cols = m->d_q + m->d_kv;
     CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, w.t_wqkv, p, m->num_sms, st));
+    prof_mark(m, VERILLM_PROF_GEMM_QKV, st);
     CU_TRY(launch_attention(m->qkv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads, c.head_dim, m->attn, st));
+    prof_mark(m, VERILLM_PROF_ATTENTION, st);
     p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
     CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_attn, w.t_wo, p, m->num_sms, st));
+    prof_mark(m, VERILLM_PROF_GEMM_O, st);
     CU_TRY(launch_rmsnorm(m->resid, w.ffn_norm, m->xn, r.M, c.d_model, c.rms_eps, st));
+    prof_mark(m, VERILLM_PROF_RMSNORM, st);
     p.N = 2 * c.d_ffn; p.K = c.d_model; p.out = m->mid; p.ldo = c.d_ffn;
     CU_TRY(launch_gemm(EPI_SWIGLU, m->t_xn, w.t_wgu, p, m->num_sms, st));
+    prof_mark(m, VERILLM_PROF_GEMM_GATE_UP, st);
     p.N = c.d_model; p.K = c.d_ffn; p.out = m->resid; p.ldo = c.d_model;
     if (r.cmp_layer) {
         p.slot_first = r.cmp_layer->slot_first; p.slot_next = r.cmp_layer->slot_next; p.n_check = r.cmp_layer->n_check;
@@ -193,6 +216,7 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
     } else {
         CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_mid, w.t_wd, p, m->num_sms, st));
     }
+    prof_mark(m, VERILLM_PROF_GEMM_DOWN, st);
     *launches += 7;
     return VERILLM_OK;
 }
@@ -258,10 +282,40 @@ void verillm_free(verillm_model* m) {
     DecodeState& d = m->dec;
     cudaFree(d.kv_cache); cudaFree(d.hidden_tmp); cudaFree(d.resid); cudaFree(d.qkv); cudaFree(d.gu);
     cudaFree(d.xn); cudaFree(d.q); cudaFree(d.attn); cudaFree(d.mid); cudaFree(d.ints);
+    for (cudaEvent_t e : m->prof.ev) cudaEventDestroy(e);
     delete m;
 }
 
 int32_t verillm_last_launch_count(const verillm_model* m) { return m ? m->last_launches : 0; }
+
+int verillm_profile_enable(verillm_model* m, int32_t on) {
+    if (!m) return VERILLM_E_INVAL;
+    Profile& p = m->prof;
+    if (on && p.ev.empty()) {
+        const size_t n = static_cast<size_t>(m->cfg.n_layers) * 7 + 8;
+        p.ev.resize(n);
+        p.cls.assign(n, -1);
+        for (size_t i = 0; i < n; ++i) CU_TRY(cudaEventCreate(&p.ev[i]));
+    }
+    p.on = on != 0;
+    p.n = 0;
+    return VERILLM_OK;
+}
+
+int verillm_profile_read(verillm_model* m, float* ms, int32_t* launches) {
+    if (!m || !ms || !launches) return VERILLM_E_INVAL;
+    Profile& p = m->prof;
+    for (int i = 0; i < VERILLM_PROF_NCLASS; ++i) { ms[i] = 0.f; launches[i] = 0; }
+    if (p.n < 2) return VERILLM_OK;
+    CU_TRY(cudaEventSynchronize(p.ev[p.n - 1]));
+    for (int i = 1; i < p.n; ++i) {
+        float t = 0.f;
+        CU_TRY(cudaEventElapsedTime(&t, p.ev[i - 1], p.ev[i]));
+        const int c = p.cls[i];
+        if (c >= 0 && c < VERILLM_PROF_NCLASS) { ms[c] += t; launches[c] += 1; }
+    }
+    return VERILLM_OK;
+}
 
 int verillm_load_layer(verillm_model* m, int32_t layer, const verillm_layer_weights* w, int32_t on_device) {
     if (!m || !w || layer < 0 || layer >= m->cfg.n_layers) return VERILLM_E_INVAL;
@@ -416,6 +470,8 @@ int verillm_verify_prefill(verillm_model* m, const int32_t* tokens, const int32_
     const verillm_config& c = m->cfg;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     int launches = 0;
+    m->prof.n = 0;
+    prof_mark(m, -1, st);
     CU_TRY(cudaMemsetAsync(rep->status, 0, sizeof(int), st));
     CU_TRY(cudaMemcpyAsync(m->cu_dev, cu_seqlens, sizeof(int) * (batch + 1), cudaMemcpyHostToDevice, st));
     if (n_check > 0) {
@@ -426,6 +482,7 @@ int verillm_verify_prefill(verillm_model* m, const int32_t* tokens, const int32_
     CU_TRY(launch_slot_lists(m->tok_of_slot, n_check, M, m->slot_first, m->slot_next, st));
     CU_TRY(launch_embed(tokens, m->embed, M, c.d_model, c.vocab, m->resid, rep->status, st));
     launches += 2 + (n_check > 0 ? 1 : 0);
+    prof_mark(m, VERILLM_PROF_SETUP, st);
 
     const size_t e_commit = commit_dtype == VERILLM_BF16 ? 2 : 4;
     GemmParams cl;
@@ -445,6 +502,7 @@ int verillm_verify_prefill(verillm_model* m, const int32_t* tokens, const int32_
     CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, m->seq_of_slot, n_check, c.n_layers, batch, rep->seq_ok,
                               rep->seq_score, st));
     launches += (n_check > 0 ? 1 : 0) + 1;
+    prof_mark(m, VERILLM_PROF_VERDICT, st);
     m->last_launches = launches;
     return VERILLM_OK;
 }
@@ -548,7 +606,6 @@ int verillm_decode_commit(verillm_model* m, const int32_t* tokens, const int32_t
     // ---------------------------------------------------------------- phase B: token-by-token decode
     // rows of step t: the sequences with n_prefill <= t < len, in batch order
     std::vector<int> step_first, row_tok, row_pos, row_start;
-    std::vector<std::vector<int>> row_of_seq_at;  // not stored: recomputed below
     int t_begin = max_len, t_end = max_len;
     for (int b = 0; b < batch; ++b) t_begin = std::min(t_begin, np[b]);
     for (int t = t_begin; t < t_end; ++t) {
