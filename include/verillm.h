@@ -180,6 +180,22 @@ int verillm_compare(const float *hidden, const void *committed, int32_t commit_d
                     int32_t n_check, int32_t d_model, const int32_t *check_seq, int32_t batch,
                     const verillm_tol *tol, const verillm_report *report, void *cuda_stream);
 
+/* Same computation, arguments and results as verillm_compare, for callers that must not allocate device
+ * memory while they run: code inside a latency-critical serving loop where cudaMalloc would synchronise
+ * the device, processes that handed their whole memory budget to a pool at start-up, and hosts that run
+ * under an allocator they cannot re-enter.  (The paper has no counterpart; this is a packaging variant.)
+ * Its scratch (the partial sums and the slot-to-sequence map) is a fixed array of about 3.3 MB inside the
+ * library, held by every GPU that loads the library until the process exits.  Limits: n_check <= 65536
+ * and n_layers * n_check <= 65536, otherwise VERILLM_E_SHAPE and nothing is launched.  The call makes no
+ * cudaMalloc / cudaFree and uses no allocating library routine.  The first call on each device looks up
+ * the array's device address (cudaGetSymbolAddress); make that first call outside any stream capture.
+ * All calls share the one array, which keeps whatever the previous call left there (the part a call reads
+ * is cleared first): two calls that overlap on the GPU, on different streams or from different threads,
+ * race on it and must be serialised by the caller. */
+int verillm_compare_noalloc(const float *hidden, const void *committed, int32_t commit_dtype, int32_t n_layers,
+                            int32_t n_check, int32_t d_model, const int32_t *check_seq, int32_t batch,
+                            const verillm_tol *tol, const verillm_report *report, void *cuda_stream);
+
 /* Single steps of the path, exposed for testing against the oracle.  All pointers DEVICE. */
 
 /* C[M][N] = A[M][K] * B[N][K]^T, bf16 inputs, fp32 accumulation on the tensor cores; out_f32 selects a

@@ -27,7 +27,7 @@ DEV_TOKEN_RANGE, DEV_WAIT_TIMEOUT = 1, 2
 
 EXPORTS = (
     "verillm_default_tol", "verillm_load_weights", "verillm_load_layer", "verillm_load_globals",
-    "verillm_verify_prefill", "verillm_decode_commit", "verillm_compare", "verillm_op_gemm",
+    "verillm_verify_prefill", "verillm_decode_commit", "verillm_compare", "verillm_compare_noalloc", "verillm_op_gemm",
     "verillm_op_rmsnorm", "verillm_op_attention", "verillm_free", "verillm_strerror",
     "verillm_last_launch_count", "verillm_profile_enable", "verillm_profile_read",
 )
@@ -106,6 +106,8 @@ def lib() -> C.CDLL:
             C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
             C.POINTER(Tol), C.POINTER(ReportC), C.c_void_p,
         ]
+        L.verillm_compare_noalloc.argtypes = L.verillm_compare.argtypes
+        L.verillm_compare_noalloc.restype = C.c_int
         L.verillm_op_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.verillm_op_rmsnorm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p]
         L.verillm_op_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
@@ -114,7 +116,7 @@ def lib() -> C.CDLL:
         L.verillm_profile_enable.restype = C.c_int
         L.verillm_profile_read.restype = C.c_int
         for name in ("verillm_load_weights", "verillm_load_layer", "verillm_load_globals", "verillm_verify_prefill",
-                     "verillm_decode_commit", "verillm_compare", "verillm_op_gemm", "verillm_op_rmsnorm",
+                     "verillm_decode_commit", "verillm_compare", "verillm_compare_noalloc", "verillm_op_gemm", "verillm_op_rmsnorm",
                      "verillm_op_attention"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -312,6 +314,25 @@ def compare(hidden: torch.Tensor, committed: torch.Tensor, check_seq: Sequence[i
         code = lib().verillm_compare(hidden.data_ptr(), committed.data_ptr(), BF16 if committed.dtype == torch.bfloat16 else F32,
                                      n_layers, n_check, d, cs.ctypes.data, batch, C.byref(tol), C.byref(st), _stream_ptr(stream))
     _check(code, "verillm_compare")
+    return rep
+
+
+def compare_noalloc(hidden: torch.Tensor, committed: torch.Tensor, check_seq: Sequence[int], batch: int,
+                    tol: Optional[Tol] = None, report: Optional[Report] = None,
+                    stream: Optional[torch.cuda.Stream] = None) -> Report:
+    """verillm_compare_noalloc: like `compare`, but the library's scratch is a fixed array inside the library,
+    so the call itself allocates nothing.  Pass a `report` made beforehand to keep this wrapper from
+    allocating the output tensors too.  Raises E_SHAPE beyond n_layers * n_check = 65536."""
+    n_layers, n_check, d = hidden.shape
+    cs = _i32(check_seq)
+    tol = tol or default_tol()
+    rep = report or Report(n_check, n_layers, batch, d, hidden.device, False)
+    st = rep.c_struct()
+    with torch.cuda.device(hidden.device):
+        code = lib().verillm_compare_noalloc(hidden.data_ptr(), committed.data_ptr(),
+                                             BF16 if committed.dtype == torch.bfloat16 else F32, n_layers, n_check, d,
+                                             cs.ctypes.data, batch, C.byref(tol), C.byref(st), _stream_ptr(stream))
+    _check(code, "verillm_compare_noalloc")
     return rep
 
 

@@ -535,6 +535,55 @@ int verillm_compare(const float* hidden, const void* committed, int32_t commit_d
     return VERILLM_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Comparison and verdict without any allocation.  The scratch that verillm_compare takes from the
+// stream-ordered allocator lives here in a fixed array that is part of the loaded library image.
+// Layout: [kNoAllocMaxRows][kNPart] floats of partial sums, then [kNoAllocMaxChecks] ints.
+constexpr int kNoAllocMaxRows = 65536;    // n_layers * n_check
+constexpr int kNoAllocMaxChecks = 65536;  // n_check
+constexpr size_t kNoAllocPartialBytes = static_cast<size_t>(kNoAllocMaxRows) * kNPart * sizeof(float);
+constexpr size_t kNoAllocBytes = kNoAllocPartialBytes + static_cast<size_t>(kNoAllocMaxChecks) * sizeof(int);
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+// Device address of the array on each device, resolved on the first call made with that device current.
+// (In host code `g_noalloc_scratch` is only a handle for the runtime, never a pointer a kernel may use.)
+static void* g_noalloc_ptr[64] = {nullptr};
+
+int verillm_compare_noalloc(const float* hidden, const void* committed, int32_t commit_dtype, int32_t n_layers,
+                            int32_t n_check, int32_t d_model, const int32_t* check_seq, int32_t batch,
+                            const verillm_tol* tol, const verillm_report* rep, void* cuda_stream) {
+    if (!hidden || !committed || !check_seq || !tol || !rep) return VERILLM_E_INVAL;
+    if (commit_dtype != VERILLM_BF16 && commit_dtype != VERILLM_F32) return VERILLM_E_INVAL;
+    if (n_layers < 1 || n_check < 1 || batch < 1) return VERILLM_E_INVAL;
+    if (d_model < 8 || d_model % 8 != 0) return VERILLM_E_SHAPE;
+    if (n_check > kNoAllocMaxChecks || static_cast<long long>(n_layers) * n_check > kNoAllocMaxRows)
+        return VERILLM_E_SHAPE;  // beyond the fixed scratch: use verillm_compare
+    if (!rep->stats || !rep->pos_ok || !rep->first_bad_layer || !rep->seq_ok || !rep->seq_score || !rep->status)
+        return VERILLM_E_INVAL;
+    for (int s = 0; s < n_check; ++s)
+        if (check_seq[s] < 0 || check_seq[s] >= batch) return VERILLM_E_RANGE;
+    int dev = 0;
+    CU_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return VERILLM_E_INVAL;
+    if (!g_noalloc_ptr[dev]) {
+        void* ptr = nullptr;
+        CU_TRY(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+        g_noalloc_ptr[dev] = ptr;
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const size_t rows = static_cast<size_t>(n_layers) * n_check;
+    float* partials = reinterpret_cast<float*>(g_noalloc_ptr[dev]);
+    int* seq_dev = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(g_noalloc_ptr[dev]) + kNoAllocPartialBytes);
+    // the array still holds the previous call's records: wipe the part this call will read
+    CU_TRY(cudaMemsetAsync(partials, 0, rows * kNPart * sizeof(float), st));
+    CU_TRY(cudaMemsetAsync(rep->status, 0, sizeof(int), st));
+    CU_TRY(cudaMemcpyAsync(seq_dev, check_seq, sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+    CU_TRY(launch_compare_rows(hidden, committed, static_cast<int>(rows), d_model, cmp_params(*tol, commit_dtype), partials, st));
+    CU_TRY(launch_verdict(partials, n_layers, n_check, 1, d_model, tol_dev(*tol), rep->status, rep->stats, rep->pos_ok,
+                          rep->first_bad_layer, st));
+    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, seq_dev, n_check, n_layers, batch, rep->seq_ok, rep->seq_score, st));
+    return VERILLM_OK;
+}
+
 int verillm_decode_commit(verillm_model* m, const int32_t* tokens, const int32_t* cu_seqlens, int32_t batch,
                           int32_t n_prefill, const int32_t* check_seq, const int32_t* check_pos, int32_t n_check,
                           void* committed_out, int32_t commit_dtype, int32_t* status, void* cuda_stream) {
