@@ -252,11 +252,13 @@ def run_ours(args, wl):
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_wall0 = time.time()
+    torch.cuda.profiler.start()  # a profiler started with --profile-from-start off sees only the timed steps
     e0.record(stream)
     for _ in range(args.steps):
         step()
     e1.record(stream)
     torch.cuda.synchronize()
+    torch.cuda.profiler.stop()
     t_wall1 = time.time()
     vdist.barrier()
     seconds = e0.elapsed_time(e1) / 1e3
@@ -367,11 +369,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="reduced depth at full width (same launches per layer; for small profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2509_24257_b200 import synth
 
     wl = synth.WORKLOADS[args.workload]
+    if args.layers > 0:
+        wl = wl.with_layers(args.layers)
     if args.impl == "reference":
         run_reference(args, wl)
     else:
