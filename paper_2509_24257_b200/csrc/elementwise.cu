@@ -143,18 +143,19 @@ __global__ void compare_rows_kernel(const float* __restrict__ hidden, const void
 }
 
 // ------------------------------------------------------------------ verdict
-// One thread per check slot: sums the column-tile partials of every layer in a fixed order, derives
-// the reported statistics, applies the enabled tests (b = 1[T_v <= tau]; a non-finite value or a
-// device-side error rejects) and records the first failing layer.
+// One warp per check slot, lanes over layers: each lane sums the column-tile partials of its layers in
+// a fixed order, derives the reported statistics and applies the enabled tests (b = 1[T_v <= tau]; a
+// non-finite value or a device-side error rejects); the first failing layer is the minimum over lanes.
 __global__ void verdict_kernel(const float* __restrict__ partials, int n_layers, int n_check, int n_tiles, int d,
                                TolDev tol, const int* __restrict__ status, float* __restrict__ stats,
                                uint8_t* __restrict__ pos_ok, int* __restrict__ first_bad_layer) {
-    const int slot = blockIdx.x * blockDim.x + threadIdx.x;
+    const int slot = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
     if (slot >= n_check) return;
     const bool dev_error = status != nullptr && *status != 0;
-    int first_bad = -1;
+    int first_bad = 0x7FFFFFFF;
     const float inv_d = 1.f / static_cast<float>(d);
-    for (int l = 0; l < n_layers; ++l) {
+    for (int l = lane; l < n_layers; l += 32) {
         const float* rec = partials + (static_cast<size_t>(l) * n_check + slot) * n_tiles * kNPart;
         float ss = 0.f, rr = 0.f, sa = 0.f, sg = 0.f, mx = 0.f;
         uint32_t n_mis = 0, n_large = 0, n_small = 0, n_exact = 0, n_q = 0, n_z = 0, n_nf = 0;
@@ -187,49 +188,52 @@ __global__ void verdict_kernel(const float* __restrict__ partials, int n_layers,
             ok = ok && (p_e < tol.pe_max) && (p_m > tol.pm_min) && (p_w > tol.pw_min) &&
                  (fabsf(mean_signed) <= tol.e_abs_max);
         }
-        if (!ok && first_bad < 0) first_bad = l;
+        if (!ok && l < first_bad) first_bad = l;
 
-        float* o = stats + (static_cast<size_t>(slot) * n_layers + l) * VERILLM_NSTAT;
-        o[VERILLM_STAT_REL_L2] = rel;
-        o[VERILLM_STAT_MAX_ABS] = mx;
-        o[VERILLM_STAT_MAE] = mae;
-        o[VERILLM_STAT_MEAN_SIGNED] = mean_signed;
-        o[VERILLM_STAT_P_E] = p_e;
-        o[VERILLM_STAT_P_M] = p_m;
-        o[VERILLM_STAT_P_W] = p_w;
-        o[VERILLM_STAT_Q_SMALL] = q_small;
-        o[VERILLM_STAT_Z_LARGE] = z_large;
-        o[VERILLM_STAT_N_EXP_MISMATCH] = static_cast<float>(n_mis);
-        o[VERILLM_STAT_N_MANT_LARGE] = static_cast<float>(n_large);
-        o[VERILLM_STAT_N_MANT_SMALL] = static_cast<float>(n_small);
-        o[VERILLM_STAT_N_EXACT] = static_cast<float>(n_exact);
-        o[VERILLM_STAT_N_NONFINITE] = static_cast<float>(n_nf);
-        o[VERILLM_STAT_L2_DELTA] = l2d;
-        o[VERILLM_STAT_L2_REF] = l2r;
+        float4* o = reinterpret_cast<float4*>(stats + (static_cast<size_t>(slot) * n_layers + l) * VERILLM_NSTAT);
+        o[0] = make_float4(rel, mx, mae, mean_signed);                       // REL_L2, MAX_ABS, MAE, MEAN_SIGNED
+        o[1] = make_float4(p_e, p_m, p_w, q_small);                          // P_E, P_M, P_W, Q_SMALL
+        o[2] = make_float4(z_large, static_cast<float>(n_mis), static_cast<float>(n_large),
+                           static_cast<float>(n_small));                     // Z_LARGE, N_EXP_MISMATCH, N_MANT_LARGE, N_MANT_SMALL
+        o[3] = make_float4(static_cast<float>(n_exact), static_cast<float>(n_nf), l2d, l2r);  // N_EXACT, N_NONFINITE, L2_*
     }
-    pos_ok[slot] = first_bad < 0 ? 1 : 0;
-    first_bad_layer[slot] = first_bad;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) first_bad = min(first_bad, __shfl_xor_sync(0xFFFFFFFFu, first_bad, o));
+    if (lane == 0) {
+        pos_ok[slot] = first_bad == 0x7FFFFFFF ? 1 : 0;
+        first_bad_layer[slot] = first_bad == 0x7FFFFFFF ? -1 : first_bad;
+    }
 }
 
-// One thread per sequence, slots visited in index order: accept iff all its checked positions were
-// accepted (one deviation above tolerance suffices to fail); score = mean MAE over its (slot, layer) cells.
+// One warp per sequence, lanes over check slots: accept iff all its checked positions were accepted (one
+// deviation above tolerance suffices to fail); score = mean MAE over its (slot, layer) cells.  Per-lane
+// double sums are combined in a fixed shuffle order, so the result is reproducible.
 __global__ void seq_verdict_kernel(const float* __restrict__ stats, const uint8_t* __restrict__ pos_ok,
                                    const int* __restrict__ seq_of_slot, int n_check, int n_layers, int batch,
                                    uint8_t* __restrict__ seq_ok, float* __restrict__ seq_score) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
     if (b >= batch) return;
-    bool ok = true;
+    int bad = 0;
     double sum = 0.0;
-    long long cells = 0;
-    for (int s = 0; s < n_check; ++s) {
+    int cells = 0;
+    for (int s = lane; s < n_check; s += 32) {
         if (seq_of_slot[s] != b) continue;
-        ok = ok && (pos_ok[s] != 0);
+        bad |= (pos_ok[s] == 0) ? 1 : 0;
         for (int l = 0; l < n_layers; ++l)
             sum += static_cast<double>(stats[(static_cast<size_t>(s) * n_layers + l) * VERILLM_NSTAT + VERILLM_STAT_MAE]);
         cells += n_layers;
     }
-    seq_ok[b] = ok ? 1 : 0;
-    seq_score[b] = cells > 0 ? static_cast<float>(sum / static_cast<double>(cells)) : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        bad |= __shfl_xor_sync(0xFFFFFFFFu, bad, o);
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+        cells += __shfl_xor_sync(0xFFFFFFFFu, cells, o);
+    }
+    if (lane == 0) {
+        seq_ok[b] = bad ? 0 : 1;
+        seq_score[b] = cells > 0 ? static_cast<float>(sum / static_cast<double>(cells)) : 0.f;
+    }
 }
 
 // ------------------------------------------------------------------ decode-side kernels
@@ -447,7 +451,7 @@ cudaError_t launch_compare_rows(const float* hidden, const void* committed, int 
 cudaError_t launch_verdict(const float* partials, int n_layers, int n_check, int n_tiles, int d, const TolDev& tol,
                            const int* status, float* stats, uint8_t* pos_ok, int* first_bad_layer, cudaStream_t s) {
     if (n_check <= 0) return cudaSuccess;
-    verdict_kernel<<<(n_check + 63) / 64, 64, 0, s>>>(partials, n_layers, n_check, n_tiles, d, tol, status, stats,
+    verdict_kernel<<<(n_check + 3) / 4, 128, 0, s>>>(partials, n_layers, n_check, n_tiles, d, tol, status, stats,
                                                       pos_ok, first_bad_layer);
     return cudaGetLastError();
 }
@@ -455,7 +459,7 @@ cudaError_t launch_verdict(const float* partials, int n_layers, int n_check, int
 cudaError_t launch_seq_verdict(const float* stats, const uint8_t* pos_ok, const int* seq_of_slot, int n_check,
                                int n_layers, int batch, uint8_t* seq_ok, float* seq_score, cudaStream_t s) {
     if (batch <= 0) return cudaSuccess;
-    seq_verdict_kernel<<<(batch + 63) / 64, 64, 0, s>>>(stats, pos_ok, seq_of_slot, n_check, n_layers, batch, seq_ok,
+    seq_verdict_kernel<<<(batch + 3) / 4, 128, 0, s>>>(stats, pos_ok, seq_of_slot, n_check, n_layers, batch, seq_ok,
                                                         seq_score);
     return cudaGetLastError();
 }

@@ -24,18 +24,19 @@ constexpr int BAR_BYTES = 256;
 constexpr int GEMM_SMEM = TILE_BYTES + BAR_BYTES + 1024;  // + slack for the 1024-byte alignment
 constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;  // two fp32 accumulators of 128 lanes x 256 columns
-constexpr int GROUP_M = 16;     // tiles are walked in bands of 16 tile-rows, row index fastest
 
 struct TileCoord {
     int m_idx, n_idx;
 };
 
-__device__ __forceinline__ TileCoord tile_coord(int tile, int num_m, int num_n) {
-    const int per_group = GROUP_M * num_n;
+// Tiles are walked in bands of `group_m` tile-rows, row index fastest, so that the CTAs of a wave share
+// weight tiles through L2 and a band's activation rows stay L2-resident across its column tiles.
+__device__ __forceinline__ TileCoord tile_coord(int tile, int num_m, int num_n, int group_m) {
+    const int per_group = group_m * num_n;
     const int g = tile / per_group;
     const int r = tile - g * per_group;
-    const int m_first = g * GROUP_M;
-    const int gm = min(GROUP_M, num_m - m_first);
+    const int m_first = g * group_m;
+    const int gm = min(group_m, num_m - m_first);
     TileCoord c;
     c.n_idx = r / gm;
     c.m_idx = m_first + (r - c.n_idx * gm);
@@ -74,8 +75,7 @@ template <int EPI>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t trow, int row, int n0, int n_idx) {
     const bool row_ok = row < p.M;
 
-    if constexpr (EPI == EPI_STORE_BF16 || EPI == EPI_STORE_F32 || EPI == EPI_RESID_ADD ||
-                  EPI == EPI_RESID_ADD_COMPARE) {
+    if constexpr (EPI == EPI_STORE_BF16 || EPI == EPI_STORE_F32) {
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
             const int col = n0 + c * 32;
@@ -85,23 +85,44 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t trow
             if (!row_ok) continue;
             if constexpr (EPI == EPI_STORE_BF16) {
                 store_bf16x32(reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<size_t>(row) * p.ldo + col, v);
-            } else if constexpr (EPI == EPI_STORE_F32) {
-                float4* d4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) +
-                                                       static_cast<size_t>(row) * p.ldo + col);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
             } else {
                 float4* d4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) +
                                                        static_cast<size_t>(row) * p.ldo + col);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    float4 r = d4[i];
-                    r.x += v[4 * i];
-                    r.y += v[4 * i + 1];
-                    r.z += v[4 * i + 2];
-                    r.w += v[4 * i + 3];
-                    d4[i] = r;
-                }
+                for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+        }
+    } else if constexpr (EPI == EPI_RESID_ADD || EPI == EPI_RESID_ADD_COMPARE) {
+        // in-place fp32 read-modify-write of the thread's row; the reads of the next 32-column chunk are
+        // issued before the current chunk is combined, so their latency overlaps the TMEM load and the stores
+        float* rrow = reinterpret_cast<float*>(p.out) + static_cast<size_t>(row_ok ? row : 0) * p.ldo + n0;
+        const int n_chunks = min(BN, p.N - n0) / 32;
+        float4 nxt[8];
+        if (row_ok && n_chunks > 0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) nxt[i] = reinterpret_cast<const float4*>(rrow)[i];
+        }
+#pragma unroll 1
+        for (int c = 0; c < n_chunks; ++c) {
+            float4 cur[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) cur[i] = nxt[i];
+            if (row_ok && c + 1 < n_chunks) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) nxt[i] = reinterpret_cast<const float4*>(rrow + (c + 1) * 32)[i];
+            }
+            float v[32];
+            load_acc(trow + c * 32, v);
+            if (!row_ok) continue;
+            float4* d4 = reinterpret_cast<float4*>(rrow + c * 32);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float4 r = cur[i];
+                r.x += v[4 * i];
+                r.y += v[4 * i + 1];
+                r.z += v[4 * i + 2];
+                r.w += v[4 * i + 3];
+                d4[i] = r;
             }
         }
     } else if constexpr (EPI == EPI_QKV_ROPE) {
@@ -240,6 +261,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int num_n = (p.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     const int num_kb = (p.K + BK - 1) / BK;
+    const int group_m = p.group_m > 0 ? p.group_m : 16;
 
     if (threadIdx.x == 0) {
         s_failed = 0;
@@ -271,7 +293,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const TileCoord tc = tile_coord(tile, num_m, num_n);
+                const TileCoord tc = tile_coord(tile, num_m, num_n, group_m);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status)) {
                         ok = false;
@@ -337,7 +359,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         uint32_t acc_phase = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-            const TileCoord tc = tile_coord(tile, num_m, num_n);
+            const TileCoord tc = tile_coord(tile, num_m, num_n, group_m);
             if (!mbar_wait(acc_full_bar(acc), acc_phase, p.status)) {
                 ok = false;
                 break;

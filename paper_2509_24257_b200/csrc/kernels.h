@@ -27,6 +27,7 @@ struct GemmParams {
     int M, N, K;
     void* out;  // bf16 / fp32 matrix or the fp32 residual stream
     int ldo;    // leading dimension of out, elements
+    int group_m;  // tile-rows per band of the tile walk (0: default 16)
     // EPI_QKV_ROPE
     const float2* rope_cs;    // [position][head_dim/2] (cos, sin)
     const int* pos_of_token;  // [M]

@@ -190,24 +190,34 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
     std::memset(&p, 0, sizeof(p));
     p.status = status;
     p.M = r.M;
+    // Activations of the K = d_model projections (M x d bf16) stay L2-resident when the band spans every
+    // tile-row, so each weight tile is fetched from HBM once; the down projection streams a wider A.
+    const int num_m = (r.M + kGemmBM - 1) / kGemmBM;
+#ifndef VL_BAND_L2_BYTES
+#define VL_BAND_L2_BYTES 0u
+#endif
+    const bool a_fits_l2 = static_cast<size_t>(r.M) * c.d_model * 2 <= VL_BAND_L2_BYTES;  // measured: bands of 16 win
+    const int band_d = a_fits_l2 ? num_m : 16;
 
     CU_TRY(launch_rmsnorm(m->resid, w.attn_norm, m->xn, r.M, c.d_model, c.rms_eps, st));
     prof_mark(m, VERILLM_PROF_RMSNORM, st);
-    p.N = m->n_qkv; p.K = c.d_model; p.out = m->qkv; p.ldo = m->n_qkv;
+    p.N = m->n_qkv; p.K = c.d_model; p.out = m->qkv; p.ldo = m->n_qkv; p.group_m = band_d;
     p.rope_cs = m->rope_cs; p.pos_of_token = m->pos_of_token; p.head_dim = c.head_dim; p.rope_cols = m->d_q + m->d_kv;
     CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, w.t_wqkv, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_QKV, st);
     CU_TRY(launch_attention(m->qkv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads, c.head_dim, m->attn, st));
     prof_mark(m, VERILLM_PROF_ATTENTION, st);
     p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
+    p.group_m = static_cast<size_t>(r.M) * m->d_q * 2 <= VL_BAND_L2_BYTES ? num_m : 16;
     CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_attn, w.t_wo, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_O, st);
     CU_TRY(launch_rmsnorm(m->resid, w.ffn_norm, m->xn, r.M, c.d_model, c.rms_eps, st));
     prof_mark(m, VERILLM_PROF_RMSNORM, st);
-    p.N = 2 * c.d_ffn; p.K = c.d_model; p.out = m->mid; p.ldo = c.d_ffn;
+    p.N = 2 * c.d_ffn; p.K = c.d_model; p.out = m->mid; p.ldo = c.d_ffn; p.group_m = band_d;
     CU_TRY(launch_gemm(EPI_SWIGLU, m->t_xn, w.t_wgu, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_GATE_UP, st);
     p.N = c.d_model; p.K = c.d_ffn; p.out = m->resid; p.ldo = c.d_model;
+    p.group_m = static_cast<size_t>(r.M) * c.d_ffn * 2 <= VL_BAND_L2_BYTES ? num_m : 16;
     if (r.cmp_layer) {
         p.slot_first = r.cmp_layer->slot_first; p.slot_next = r.cmp_layer->slot_next; p.n_check = r.cmp_layer->n_check;
         p.committed = r.cmp_layer->committed; p.partials = r.cmp_layer->partials; p.hidden_out = r.cmp_layer->hidden_out;
