@@ -1,0 +1,305 @@
+// Causal grouped-query attention over packed sequences on the fifth-generation tensor cores:
+// softmax(q k^T / sqrt(dh) + causal mask) v, flash style ("a single forward pass under the causal mask").
+//
+// One CTA owns 128 query rows of one (sequence, query head) and walks the key/value tiles of 64 positions
+// up to the diagonal.  Warp 4 (one thread) drives everything asynchronous: TMA loads of Q and of a
+// double-buffered K/V ring (128-byte swizzle), S = Q K^T and O_blk = P V as tcgen05.mma into tensor
+// memory.  Warps 0-3 own one query row per thread: they read S from TMEM, keep the online softmax
+// (running maximum and sum, fp32, exp2) in registers, write P as bf16 into shared memory in the operand
+// layout of the second product, and fold each O_blk into their fp32 output row.  S is double-buffered, so
+// Q K^T of the next tile overlaps the softmax of the current one; two CTAs share an SM, so one CTA's
+// tensor work overlaps the other's softmax.  V is consumed as it lies in memory ([key][dh], an MN-major
+// B operand).  Every wait is bounded; on a timeout the CTA records the error, drains and frees its TMEM.
+#include "kernels.h"
+
+namespace vl {
+
+namespace {
+
+constexpr int TC_BM = 128;
+constexpr int TC_BN = 64;
+constexpr int TC_THREADS = 160;
+constexpr int TC_TMEM_COLS = 256;  // S0 [0,64), S1 [64,128), O_blk [128, 128 + dh)
+
+template <int DH>
+struct TcSmem {
+    static constexpr uint32_t Q_BYTES = TC_BM * DH * 2;
+    static constexpr uint32_t KV_BYTES = TC_BN * DH * 2;
+    static constexpr uint32_t P_BYTES = TC_BM * TC_BN * 2;
+    static constexpr uint32_t K_OFF = Q_BYTES;
+    static constexpr uint32_t V_OFF = K_OFF + 2 * KV_BYTES;
+    static constexpr uint32_t P_OFF = V_OFF + 2 * KV_BYTES;
+    static constexpr uint32_t BAR_OFF = P_OFF + P_BYTES;
+    static constexpr uint32_t TOTAL = BAR_OFF + 128;
+};
+
+// K-major operand whose rows are 128 bytes (64 bf16) with the 128-byte swizzle: see umma_desc_k_sw128.
+// MN-major operand (V as stored: [key][dh]): 64 dh-columns contiguous per key row of 128 bytes, 8 key rows
+// per 1024-byte swizzle atom; `lbo_bytes` separates the 64-column blocks of a wider head.
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t tile_smem, uint32_t lbo_bytes) {
+    const uint64_t lo = static_cast<uint64_t>((tile_smem & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(lbo_bytes >> 4) << 16);
+    const uint64_t hi = static_cast<uint64_t>(1024u >> 4) | (1ull << 14) | (2ull << 29);
+    return lo | (hi << 32);
+}
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int DH>
+__global__ void __launch_bounds__(TC_THREADS, 2)
+attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
+               const int* __restrict__ cu_seqlens, int n_heads, int n_kv_heads, __nv_bfloat16* __restrict__ out,
+               int* status) {
+    using L = TcSmem<DH>;
+    constexpr int QB = DH / 64;  // 64-column blocks per head
+    extern __shared__ __align__(1024) uint8_t tc_smem[];
+
+    const int seq = blockIdx.z, head = blockIdx.y;
+    const int seq_start = cu_seqlens[seq];
+    const int len = cu_seqlens[seq + 1] - seq_start;
+    const int qb = static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x);  // longest rows first
+    const int q0 = qb * TC_BM;
+    if (q0 >= len) return;
+    const uint32_t sbase = smem_u32(tc_smem);
+    if ((sbase & 1023u) != 0u) {  // the swizzled tiles need a 1024-byte aligned base
+        if (threadIdx.x == 0 && status) atomicCAS(status, 0, VERILLM_DEV_WAIT_TIMEOUT);
+        return;
+    }
+    const int kvh = head * n_kv_heads / n_heads;
+    const int dq = n_heads * DH, dkv = n_kv_heads * DH;
+    const int last_row = min(q0 + TC_BM, len) - 1;
+    const int nb = last_row / TC_BN + 1;  // causal: key tiles up to the last valid row
+
+    const uint32_t q_s = sbase;
+    auto k_s = [&](int b) { return sbase + L::K_OFF + b * L::KV_BYTES; };
+    auto v_s = [&](int b) { return sbase + L::V_OFF + b * L::KV_BYTES; };
+    const uint32_t p_s = sbase + L::P_OFF;
+    const uint32_t bar = sbase + L::BAR_OFF;
+    const uint32_t q_full = bar, p_ready = bar + 8, o_full = bar + 16;
+    auto kv_full = [&](int b) { return bar + 24 + 8 * b; };
+    auto kv_empty = [&](int b) { return bar + 40 + 8 * b; };
+    auto s_full = [&](int b) { return bar + 56 + 8 * b; };
+    const uint32_t tmem_slot = bar + 72;
+    volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(tc_smem + L::BAR_OFF + 72);
+    volatile int* failed = reinterpret_cast<volatile int*>(tc_smem + L::BAR_OFF + 76);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        *failed = 0;
+        mbar_init(q_full, 1);
+        mbar_init(p_ready, 128);
+        mbar_init(o_full, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(kv_full(b), 1);
+            mbar_init(kv_empty(b), 1);
+            mbar_init(s_full(b), 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 4) {
+        tmem_alloc(tmem_slot, TC_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_ptr;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ TMA + MMA driver (one thread)
+        if (lane == 0) {
+            bool ok = true;
+            auto load_kv = [&](int j) {
+                const int b = j & 1;
+                mbar_arrive_expect_tx(kv_full(b), 2 * L::KV_BYTES);
+#pragma unroll
+                for (int c = 0; c < QB; ++c) {
+                    tma_load_2d(k_s(b) + c * (TC_BN * 128), &tmap_kv, dq + kvh * DH + c * 64, seq_start + j * TC_BN, kv_full(b));
+                    tma_load_2d(v_s(b) + c * (TC_BN * 128), &tmap_kv, dq + dkv + kvh * DH + c * 64, seq_start + j * TC_BN, kv_full(b));
+                }
+            };
+            auto issue_qk = [&](int j) {  // S[j & 1] = Q K_j^T : M 128, N 64, K = DH
+                const int b = j & 1;
+                constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, TC_BN);
+#pragma unroll
+                for (int kk = 0; kk < DH / 16; ++kk) {
+                    const uint64_t a = umma_desc_k_sw128(q_s + (kk / 4) * (TC_BM * 128)) + 2u * (kk % 4);
+                    const uint64_t bd = umma_desc_k_sw128(k_s(b) + (kk / 4) * (TC_BN * 128)) + 2u * (kk % 4);
+                    umma_bf16(tmem_base + static_cast<uint32_t>(b * TC_BN), a, bd, idesc, kk != 0 ? 1u : 0u);
+                }
+                umma_commit(s_full(b));
+            };
+            mbar_arrive_expect_tx(q_full, L::Q_BYTES);
+#pragma unroll
+            for (int c = 0; c < QB; ++c) tma_load_2d(q_s + c * (TC_BM * 128), &tmap_q, head * DH + c * 64, seq_start + q0, q_full);
+            load_kv(0);
+            if (nb > 1) load_kv(1);
+            ok = mbar_wait(q_full, 0, status) && mbar_wait(kv_full(0), 0, status);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0);
+            }
+            for (int j = 0; j < nb && ok; ++j) {
+                const int b = j & 1;
+                if (j + 1 < nb) {
+                    if (!mbar_wait(kv_full(b ^ 1), ((j + 1) >> 1) & 1, status)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_qk(j + 1);
+                }
+                if (!mbar_wait(p_ready, j & 1, status)) { ok = false; break; }
+                tc_fence_after();
+                {   // O_blk = P V_j : M 128, N = DH, K = 64 keys; V is the MN-major B operand
+                    constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, DH) | (1u << 16);
+#pragma unroll
+                    for (int kk = 0; kk < TC_BN / 16; ++kk) {
+                        const uint64_t a = umma_desc_k_sw128(p_s) + 2u * kk;
+                        const uint64_t bd = umma_desc_mn_sw128(v_s(b) + kk * 2048, TC_BN * 128);
+                        umma_bf16(tmem_base + 128u, a, bd, idesc, kk != 0 ? 1u : 0u);
+                    }
+                }
+                umma_commit(o_full);
+                umma_commit(kv_empty(b));
+                if (j + 2 < nb) {
+                    if (!mbar_wait(kv_empty(b), (j >> 1) & 1, status)) { ok = false; break; }
+                    load_kv(j + 2);
+                }
+            }
+            if (!ok) *failed = 1;
+        }
+    } else {
+        // ------------------------------------------------------------ softmax / output warps: one row per thread
+        const int r = warp * 32 + lane;
+        const int row = q0 + r;  // position inside the sequence
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+        const float scale_log2 = rsqrtf(static_cast<float>(DH)) * 1.4426950408889634f;
+        float o[DH];
+#pragma unroll
+        for (int i = 0; i < DH; ++i) o[i] = 0.f;
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int j = 0; j < nb; ++j) {
+            const int b = j & 1;
+            if (!mbar_wait(s_full(b), (j >> 1) & 1, status)) { ok = false; break; }
+            tc_fence_after();
+            const int key0 = j * TC_BN;
+            const bool need_mask = key0 + TC_BN - 1 > q0;  // uniform over the CTA
+            const uint32_t s_addr = lane_base + static_cast<uint32_t>(b * TC_BN);
+            // pass 1: row maximum of the scaled, masked scores
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < TC_BN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(s_addr + c * 32, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    float x = __uint_as_float(v[i]) * scale_log2;
+                    if (need_mask && key0 + c * 32 + i > row) x = -INFINITY;
+                    mx = fmaxf(mx, x);
+                }
+            }
+            const float m_new = fmaxf(m_run, mx);  // tile 0 holds key 0 <= row: finite from the first tile on
+            const float corr = ex2(m_run - m_new);
+            // pass 2: probabilities, row sum, bf16 P into the swizzled K-major operand tile
+            float rs = 0.f;
+#pragma unroll
+            for (int c = 0; c < TC_BN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(s_addr + c * 32, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    float pv[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        float x = __uint_as_float(v[8 * q + i]) * scale_log2 - m_new;
+                        if (need_mask && key0 + c * 32 + 8 * q + i > row) x = -INFINITY;
+                        pv[i] = ex2(x);
+                        rs += pv[i];
+                    }
+                    const int chunk = c * 4 + q;  // 16-byte chunk = 8 keys
+                    const uint32_t addr = p_s + static_cast<uint32_t>(r * 128 + ((chunk ^ (r & 7)) << 4));
+                    const uint32_t w0 = pack_bf16(pv[0], pv[1]), w1 = pack_bf16(pv[2], pv[3]);
+                    const uint32_t w2 = pack_bf16(pv[4], pv[5]), w3 = pack_bf16(pv[6], pv[7]);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3)
+                                 : "memory");
+                }
+            }
+            l_run = l_run * corr + rs;
+            m_run = m_new;
+            fence_proxy_async_smem();  // P must be visible to the tensor core's reads
+            tc_fence_before();
+            mbar_arrive(p_ready);
+            if (!mbar_wait(o_full, j & 1, status)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < DH / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(lane_base + 128u + c * 32, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], corr, __uint_as_float(v[i]));
+            }
+            tc_fence_before();
+        }
+        if (!ok) *failed = 1;
+        if (ok && row < len) {
+            const float inv = 1.f / l_run;
+            uint4* dst = reinterpret_cast<uint4*>(out + static_cast<size_t>(seq_start + row) * dq + head * DH);
+#pragma unroll
+            for (int q = 0; q < DH / 8; ++q) {
+                uint4 u;
+                u.x = pack_bf16(o[8 * q + 0] * inv, o[8 * q + 1] * inv);
+                u.y = pack_bf16(o[8 * q + 2] * inv, o[8 * q + 3] * inv);
+                u.z = pack_bf16(o[8 * q + 4] * inv, o[8 * q + 5] * inv);
+                u.w = pack_bf16(o[8 * q + 6] * inv, o[8 * q + 7] * inv);
+                dst[q] = u;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*failed) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {
+        }
+        __syncthreads();
+    }
+    if (warp == 4) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TC_TMEM_COLS);
+    }
+}
+
+}  // namespace
+
+cudaError_t attention_tc_init() {
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(TcSmem<64>::TOTAL));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                static_cast<int>(TcSmem<128>::TOTAL));
+}
+
+cudaError_t launch_attention_tc(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, const int* cu_seqlens_dev,
+                                int batch, int max_seqlen, int n_heads, int n_kv_heads, int head_dim, void* out,
+                                int* status, cudaStream_t stream) {
+    if (batch <= 0 || max_seqlen <= 0) return cudaSuccess;
+    const dim3 grid((max_seqlen + TC_BM - 1) / TC_BM, n_heads, batch);
+    __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out);
+    if (head_dim == 64)
+        attn_tc_kernel<64><<<grid, TC_THREADS, TcSmem<64>::TOTAL, stream>>>(tmap_q, tmap_kv, cu_seqlens_dev, n_heads,
+                                                                           n_kv_heads, o, status);
+    else if (head_dim == 128)
+        attn_tc_kernel<128><<<grid, TC_THREADS, TcSmem<128>::TOTAL, stream>>>(tmap_q, tmap_kv, cu_seqlens_dev, n_heads,
+                                                                             n_kv_heads, o, status);
+    else
+        return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+}  // namespace vl

@@ -68,6 +68,7 @@ struct verillm_model {
     float* partials = nullptr;
     float2* rope_cs = nullptr;
     CUtensorMap t_xn, t_attn, t_mid;
+    CUtensorMap t_qkv_q, t_qkv_kv;  // attention operands: boxes of 128 query rows / 64 key rows
     DecodeState dec;
     Profile prof;
     int last_launches = 0;
@@ -94,6 +95,7 @@ int ensure_init() {
     if (prop.major != 10) return VERILLM_E_ARCH;
     CU_TRY(gemm_init());
     CU_TRY(attention_init());
+    CU_TRY(attention_tc_init());
     done[dev] = true;
     return VERILLM_OK;
 }
@@ -205,7 +207,12 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
     p.rope_cs = m->rope_cs; p.pos_of_token = m->pos_of_token; p.head_dim = c.head_dim; p.rope_cols = m->d_q + m->d_kv;
     CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, w.t_wqkv, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_QKV, st);
+#ifdef VL_ATTN_LEGACY
     CU_TRY(launch_attention(m->qkv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads, c.head_dim, m->attn, st));
+#else
+    CU_TRY(launch_attention_tc(m->t_qkv_q, m->t_qkv_kv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads,
+                               c.head_dim, m->attn, status, st));
+#endif
     prof_mark(m, VERILLM_PROF_ATTENTION, st);
     p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
     p.group_m = static_cast<size_t>(r.M) * m->d_q * 2 <= VL_BAND_L2_BYTES ? num_m : 16;
@@ -415,6 +422,11 @@ int verillm_load_weights(const verillm_config* cfg, const verillm_weights* weigh
     TRY_RC(dev_alloc(&m->partials, static_cast<size_t>(c.n_layers) * NC * m->n_tiles_d * kNPart));
     TRY_RC(dev_alloc(&m->rope_cs, T * (c.head_dim / 2)));
 
+    // Rows past a call's last token are never stored, but tiles that straddle the end are read: keep them finite.
+    cudaMemset(m->xn, 0, T * d * sizeof(bf16));
+    cudaMemset(m->qkv, 0, T * m->n_qkv * sizeof(bf16));
+    cudaMemset(m->attn, 0, T * m->d_q * sizeof(bf16));
+    cudaMemset(m->mid, 0, T * c.d_ffn * sizeof(bf16));
     // rotary table: angle = pos * base^(-2i/dh), evaluated in double, stored as (cos, sin) float pairs
     {
         const int half = c.head_dim / 2;
@@ -438,6 +450,8 @@ int verillm_load_weights(const verillm_config* cfg, const verillm_weights* weigh
     ok = ok && make_tmap_bf16_2d(&m->t_xn, m->xn, T, d, d, kGemmBM) == 0;
     ok = ok && make_tmap_bf16_2d(&m->t_attn, m->attn, T, m->d_q, m->d_q, kGemmBM) == 0;
     ok = ok && make_tmap_bf16_2d(&m->t_mid, m->mid, T, c.d_ffn, c.d_ffn, kGemmBM) == 0;
+    ok = ok && make_tmap_bf16_2d(&m->t_qkv_q, m->qkv, T, m->n_qkv, m->n_qkv, 128) == 0;
+    ok = ok && make_tmap_bf16_2d(&m->t_qkv_kv, m->qkv, T, m->n_qkv, m->n_qkv, 64) == 0;
     for (LayerDev& L : m->layers) {
         ok = ok && make_tmap_bf16_2d(&L.t_wqkv, L.wqkv, m->n_qkv, d, d, kGemmBN) == 0;
         ok = ok && make_tmap_bf16_2d(&L.t_wo, L.wo, d, m->d_q, m->d_q, kGemmBN) == 0;
@@ -780,8 +794,17 @@ int verillm_op_attention(const void* qkv, const int32_t* cu_seqlens, int32_t bat
         return VERILLM_E_SHAPE;
     int rc = ensure_init();
     if (rc) return rc;
+#ifdef VL_ATTN_LEGACY
     CU_TRY(launch_attention(qkv, cu_seqlens, batch, max_seqlen, n_heads, n_kv_heads, head_dim, out,
                             reinterpret_cast<cudaStream_t>(cuda_stream)));
+#else
+    const int n_qkv = (n_heads + 2 * n_kv_heads) * head_dim;
+    CUtensorMap tq, tkv;
+    if (make_tmap_bf16_2d(&tq, qkv, M, n_qkv, n_qkv, 128) != 0) return VERILLM_E_CUDA;
+    if (make_tmap_bf16_2d(&tkv, qkv, M, n_qkv, n_qkv, 64) != 0) return VERILLM_E_CUDA;
+    CU_TRY(launch_attention_tc(tq, tkv, cu_seqlens, batch, max_seqlen, n_heads, n_kv_heads, head_dim, out, nullptr,
+                               reinterpret_cast<cudaStream_t>(cuda_stream)));
+#endif
     return VERILLM_OK;
 }
 
