@@ -3,13 +3,15 @@
 //
 // One CTA owns 128 query rows of one (sequence, query head) and walks the key/value tiles of 64 positions
 // up to the diagonal.  Warp 4 (one thread) drives everything asynchronous: TMA loads of Q and of a
-// double-buffered K/V ring (128-byte swizzle), S = Q K^T and O_blk = P V as tcgen05.mma into tensor
-// memory.  Warps 0-3 own one query row per thread: they read S from TMEM, keep the online softmax
-// (running maximum and sum, fp32, exp2) in registers, write P as bf16 into shared memory in the operand
-// layout of the second product, and fold each O_blk into their fp32 output row.  S is double-buffered, so
-// Q K^T of the next tile overlaps the softmax of the current one; two CTAs share an SM, so one CTA's
-// tensor work overlaps the other's softmax.  V is consumed as it lies in memory ([key][dh], an MN-major
-// B operand).  Every wait is bounded; on a timeout the CTA records the error, drains and frees its TMEM.
+// double-buffered K/V ring (128-byte swizzle), S = Q K^T and O += P V as tcgen05.mma into tensor memory.
+// Warps 0-3 own one query row per thread: they read S from TMEM, keep the online softmax (reference
+// maximum and running sum, fp32, exp2) in registers and write P as packed bf16 back over the S columns,
+// from where the second product takes it as its A operand.  O accumulates in TMEM across tiles; it is
+// rescaled only when a row's maximum has grown by more than 2^8 since the reference maximum was taken
+// (probabilities stay below 256, the normalisation by the running sum cancels the stale reference), so
+// the softmax of tile j+1 overlaps P V of tile j, and Q K^T runs one tile ahead (two S buffers).  Two CTAs
+// share an SM.  V is consumed as it lies in memory ([key][dh], an MN-major B operand).  Every wait is
+// bounded; on a timeout the CTA records the error, drains and frees its TMEM.
 #include "kernels.h"
 
 namespace vl {
@@ -19,17 +21,16 @@ namespace {
 constexpr int TC_BM = 128;
 constexpr int TC_BN = 64;
 constexpr int TC_THREADS = 160;
-constexpr int TC_TMEM_COLS = 256;  // S0 [0,64), S1 [64,128), O_blk [128, 128 + dh)
+constexpr int TC_TMEM_COLS = 256;  // S0/P0 [0,64), S1/P1 [64,128), O [128, 128 + dh)
+constexpr float TC_RESCALE_LOG2 = 8.f;  // rescale O when a row maximum exceeds its reference by this (log2)
 
 template <int DH>
 struct TcSmem {
     static constexpr uint32_t Q_BYTES = TC_BM * DH * 2;
     static constexpr uint32_t KV_BYTES = TC_BN * DH * 2;
-    static constexpr uint32_t P_BYTES = TC_BM * TC_BN * 2;
     static constexpr uint32_t K_OFF = Q_BYTES;
     static constexpr uint32_t V_OFF = K_OFF + 2 * KV_BYTES;
-    static constexpr uint32_t P_OFF = V_OFF + 2 * KV_BYTES;
-    static constexpr uint32_t BAR_OFF = P_OFF + P_BYTES;
+    static constexpr uint32_t BAR_OFF = V_OFF + 2 * KV_BYTES;
     static constexpr uint32_t TOTAL = BAR_OFF + 128;
 };
 
@@ -76,23 +77,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const uint32_t q_s = sbase;
     auto k_s = [&](int b) { return sbase + L::K_OFF + b * L::KV_BYTES; };
     auto v_s = [&](int b) { return sbase + L::V_OFF + b * L::KV_BYTES; };
-    const uint32_t p_s = sbase + L::P_OFF;
     const uint32_t bar = sbase + L::BAR_OFF;
-    const uint32_t q_full = bar, p_ready = bar + 8, o_full = bar + 16;
-    auto kv_full = [&](int b) { return bar + 24 + 8 * b; };
-    auto kv_empty = [&](int b) { return bar + 40 + 8 * b; };
-    auto s_full = [&](int b) { return bar + 56 + 8 * b; };
-    const uint32_t tmem_slot = bar + 72;
-    volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(tc_smem + L::BAR_OFF + 72);
-    volatile int* failed = reinterpret_cast<volatile int*>(tc_smem + L::BAR_OFF + 76);
+    const uint32_t q_full = bar, o_done = bar + 8;
+    auto p_ready = [&](int b) { return bar + 16 + 8 * b; };
+    auto kv_full = [&](int b) { return bar + 32 + 8 * b; };
+    auto kv_empty = [&](int b) { return bar + 48 + 8 * b; };
+    auto s_full = [&](int b) { return bar + 64 + 8 * b; };
+    const uint32_t tmem_slot = bar + 80;
+    volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(tc_smem + L::BAR_OFF + 80);
+    volatile int* failed = reinterpret_cast<volatile int*>(tc_smem + L::BAR_OFF + 84);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         *failed = 0;
         mbar_init(q_full, 1);
-        mbar_init(p_ready, 128);
-        mbar_init(o_full, 1);
+        mbar_init(o_done, 1);
         for (int b = 0; b < 2; ++b) {
+            mbar_init(p_ready(b), 128);
             mbar_init(kv_full(b), 1);
             mbar_init(kv_empty(b), 1);
             mbar_init(s_full(b), 1);
@@ -149,18 +150,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     tc_fence_after();
                     issue_qk(j + 1);
                 }
-                if (!mbar_wait(p_ready, j & 1, status)) { ok = false; break; }
+                if (!mbar_wait(p_ready(b), (j >> 1) & 1, status)) { ok = false; break; }
                 tc_fence_after();
-                {   // O_blk = P V_j : M 128, N = DH, K = 64 keys; V is the MN-major B operand
+                {   // O (+)= P V_j : M 128, N = DH, K = 64 keys; P from TMEM (8 packed columns per 16 keys),
+                    // V is the MN-major B operand
                     constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, DH) | (1u << 16);
 #pragma unroll
                     for (int kk = 0; kk < TC_BN / 16; ++kk) {
-                        const uint64_t a = umma_desc_k_sw128(p_s) + 2u * kk;
                         const uint64_t bd = umma_desc_mn_sw128(v_s(b) + kk * 2048, TC_BN * 128);
-                        umma_bf16(tmem_base + 128u, a, bd, idesc, kk != 0 ? 1u : 0u);
+                        umma_bf16_ts(tmem_base + 128u, tmem_base + static_cast<uint32_t>(b * TC_BN + kk * 8), bd, idesc,
+                                     (j | kk) != 0 ? 1u : 0u);
                     }
                 }
-                umma_commit(o_full);
+                umma_commit(o_done);
                 umma_commit(kv_empty(b));
                 if (j + 2 < nb) {
                     if (!mbar_wait(kv_empty(b), (j >> 1) & 1, status)) { ok = false; break; }
@@ -174,11 +176,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const int r = warp * 32 + lane;
         const int row = q0 + r;  // position inside the sequence
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+        const uint32_t o_addr = lane_base + 128u;
         const float scale_log2 = rsqrtf(static_cast<float>(DH)) * 1.4426950408889634f;
-        float o[DH];
-#pragma unroll
-        for (int i = 0; i < DH; ++i) o[i] = 0.f;
-        float m_run = -INFINITY, l_run = 0.f;
+        float m_ref = -INFINITY, l_run = 0.f;
         bool ok = true;
         for (int j = 0; j < nb; ++j) {
             const int b = j & 1;
@@ -187,76 +187,85 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             const int key0 = j * TC_BN;
             const bool need_mask = key0 + TC_BN - 1 > q0;  // uniform over the CTA
             const uint32_t s_addr = lane_base + static_cast<uint32_t>(b * TC_BN);
-            // pass 1: row maximum of the scaled, masked scores
+            uint32_t v0[32], v1[32];
+            tmem_ld32(s_addr, v0);
+            tmem_ld32(s_addr + 32, v1);
+            tmem_ld_wait();
             float mx = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < TC_BN / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(s_addr + c * 32, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    float x = __uint_as_float(v[i]) * scale_log2;
-                    if (need_mask && key0 + c * 32 + i > row) x = -INFINITY;
-                    mx = fmaxf(mx, x);
+            for (int i = 0; i < 32; ++i) {
+                float x0 = __uint_as_float(v0[i]) * scale_log2, x1 = __uint_as_float(v1[i]) * scale_log2;
+                if (need_mask) {
+                    if (key0 + i > row) x0 = -INFINITY;
+                    if (key0 + 32 + i > row) x1 = -INFINITY;
                 }
+                v0[i] = __float_as_uint(x0);
+                v1[i] = __float_as_uint(x1);
+                mx = fmaxf(mx, fmaxf(x0, x1));
             }
-            const float m_new = fmaxf(m_run, mx);  // tile 0 holds key 0 <= row: finite from the first tile on
-            const float corr = ex2(m_run - m_new);
-            // pass 2: probabilities, row sum, bf16 P into the swizzled K-major operand tile
-            float rs = 0.f;
+            if (j == 0) {
+                m_ref = mx;  // tile 0 holds key 0 <= row: finite
+            } else {
+                const bool grow = mx > m_ref + TC_RESCALE_LOG2;
+                if (__any_sync(0xFFFFFFFFu, grow)) {
+                    // O holds tiles 0..j-1 relative to the old reference: wait for P V_{j-1}, then rescale
+                    const float corr = grow ? ex2(m_ref - mx) : 1.f;
+                    if (!mbar_wait(o_done, (j - 1) & 1, status)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c = 0; c < DH / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(o_addr + c * 32, o);
+                        tmem_ld_wait();
 #pragma unroll
-            for (int c = 0; c < TC_BN / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(s_addr + c * 32, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    float pv[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        float x = __uint_as_float(v[8 * q + i]) * scale_log2 - m_new;
-                        if (need_mask && key0 + c * 32 + 8 * q + i > row) x = -INFINITY;
-                        pv[i] = ex2(x);
-                        rs += pv[i];
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
+                        tmem_st32(o_addr + c * 32, o);
                     }
-                    const int chunk = c * 4 + q;  // 16-byte chunk = 8 keys
-                    const uint32_t addr = p_s + static_cast<uint32_t>(r * 128 + ((chunk ^ (r & 7)) << 4));
-                    const uint32_t w0 = pack_bf16(pv[0], pv[1]), w1 = pack_bf16(pv[2], pv[3]);
-                    const uint32_t w2 = pack_bf16(pv[4], pv[5]), w3 = pack_bf16(pv[6], pv[7]);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3)
-                                 : "memory");
+                    tmem_st_wait();
+                    l_run *= corr;
+                    if (grow) m_ref = mx;
                 }
             }
-            l_run = l_run * corr + rs;
-            m_run = m_new;
-            fence_proxy_async_smem();  // P must be visible to the tensor core's reads
-            tc_fence_before();
-            mbar_arrive(p_ready);
-            if (!mbar_wait(o_full, j & 1, status)) { ok = false; break; }
-            tc_fence_after();
+            // probabilities relative to the reference maximum, packed bf16 over the first 32 S columns
+            float rs = 0.f;
+            uint32_t pk[32];
 #pragma unroll
-            for (int c = 0; c < DH / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(lane_base + 128u + c * 32, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], corr, __uint_as_float(v[i]));
+            for (int i = 0; i < 16; ++i) {
+                const float a0 = ex2(__uint_as_float(v0[2 * i]) - m_ref), a1 = ex2(__uint_as_float(v0[2 * i + 1]) - m_ref);
+                const float b0 = ex2(__uint_as_float(v1[2 * i]) - m_ref), b1 = ex2(__uint_as_float(v1[2 * i + 1]) - m_ref);
+                rs += (a0 + a1) + (b0 + b1);
+                pk[i] = pack_bf16(a0, a1);
+                pk[16 + i] = pack_bf16(b0, b1);
             }
+            l_run += rs;
+            tmem_st32(s_addr, pk);
+            tmem_st_wait();
             tc_fence_before();
+            mbar_arrive(p_ready(b));
         }
+        if (ok && !mbar_wait(o_done, (nb - 1) & 1, status)) ok = false;
         if (!ok) *failed = 1;
-        if (ok && row < len) {
+        if (ok) {
+            tc_fence_after();
             const float inv = 1.f / l_run;
-            uint4* dst = reinterpret_cast<uint4*>(out + static_cast<size_t>(seq_start + row) * dq + head * DH);
+            __nv_bfloat16* dst = out + static_cast<size_t>(seq_start + (row < len ? row : 0)) * dq + head * DH;
+#pragma unroll 1
+            for (int c = 0; c < DH / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(o_addr + c * 32, o);
+                tmem_ld_wait();
+                if (row < len) {
 #pragma unroll
-            for (int q = 0; q < DH / 8; ++q) {
-                uint4 u;
-                u.x = pack_bf16(o[8 * q + 0] * inv, o[8 * q + 1] * inv);
-                u.y = pack_bf16(o[8 * q + 2] * inv, o[8 * q + 3] * inv);
-                u.z = pack_bf16(o[8 * q + 4] * inv, o[8 * q + 5] * inv);
-                u.w = pack_bf16(o[8 * q + 6] * inv, o[8 * q + 7] * inv);
-                dst[q] = u;
+                    for (int q = 0; q < 4; ++q) {
+                        uint4 u;
+                        u.x = pack_bf16(__uint_as_float(o[8 * q + 0]) * inv, __uint_as_float(o[8 * q + 1]) * inv);
+                        u.y = pack_bf16(__uint_as_float(o[8 * q + 2]) * inv, __uint_as_float(o[8 * q + 3]) * inv);
+                        u.z = pack_bf16(__uint_as_float(o[8 * q + 4]) * inv, __uint_as_float(o[8 * q + 5]) * inv);
+                        u.w = pack_bf16(__uint_as_float(o[8 * q + 6]) * inv, __uint_as_float(o[8 * q + 7]) * inv);
+                        reinterpret_cast<uint4*>(dst + c * 32)[q] = u;
+                    }
+                }
+                __syncwarp();
             }
         }
     }
