@@ -221,6 +221,13 @@ _WEIGHT_STD = 0.02
 _GAMMA_STD = 0.1  # norm gains are 1 + 0.1 * N(0,1): a dropped or misplaced gain must show up in parity
 
 
+def weight_std(shape: ModelShape) -> float:
+    """Std of the projection weights: 0.02 at d_model = 256, carried to wider models at constant gain
+    std * sqrt(d_model) = 0.32.  (A plain 0.02 at d_model = 4096 has gain 1.28 per projection: such a
+    random network amplifies rounding noise from layer to layer, unlike the trained models it stands for.)"""
+    return _WEIGHT_STD * math.sqrt(256.0 / max(shape.d_model, 256))
+
+
 def layer_tensor_shapes(shape: ModelShape) -> Dict[str, Tuple[int, ...]]:
     """Shapes of one layer's tensors; every projection is [out_features, in_features] row-major."""
     d, f = shape.d_model, shape.d_ffn
@@ -239,7 +246,7 @@ def layer_weights(
         if name.endswith("norm"):
             out[name] = normal_tensor(wl.seed, uid, shp, _GAMMA_STD, 1.0, device, dtype)
         else:
-            out[name] = normal_tensor(wl.seed, uid, shp, _WEIGHT_STD, 0.0, device, dtype)
+            out[name] = normal_tensor(wl.seed, uid, shp, weight_std(wl.shape), 0.0, device, dtype)
     return out
 
 
