@@ -243,6 +243,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             tc_fence_before();
             mbar_arrive(p_ready(b));
         }
+        // The last P V must have landed before O is read.  A parity wait can only tell apart the current
+        // phase and the one before it, and so far only P V_{nb-3} is known to be complete (Q K^T of the last
+        // tile was issued ahead of P V_{nb-2}): wait for the phases one at a time.
+        if (ok && nb >= 2 && !mbar_wait(o_done, (nb - 2) & 1, status)) ok = false;
         if (ok && !mbar_wait(o_done, (nb - 1) & 1, status)) ok = false;
         if (!ok) *failed = 1;
         if (ok) {

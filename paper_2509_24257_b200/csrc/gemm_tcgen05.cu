@@ -398,6 +398,220 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// CTA-pair variant: two CTAs on neighbouring SMs (a cluster of two) share one 256 x 256 output tile.
+// Each CTA stages only its 128 rows of A and its 128-row half of B per K step (32 KiB instead of 48),
+// the leader's MMA thread issues tcgen05.mma.cta_group::2 over both CTAs' shared memory and each CTA's
+// TMEM receives its own 128 rows of the accumulator.  Per unit of math this cuts the L2 -> SM traffic
+// by a third and leaves room for a 6-stage ring.  Barrier protocol: both CTAs' TMA loads count on the
+// leader's full barrier; the leader's tcgen05.commit releases the stage / publishes the accumulator in
+// both CTAs; the epilogue warps of both CTAs report the accumulator drained on the leader's barrier.
+#ifndef VL_PAIR_STAGES
+#define VL_PAIR_STAGES 6
+#endif
+constexpr int P_STAGES = VL_PAIR_STAGES;
+constexpr int P_B_STAGE_BYTES = 128 * BK * 2;  // half of the B tile
+constexpr int P_STAGE_BYTES = A_STAGE_BYTES + P_B_STAGE_BYTES;
+constexpr int P_TILE_BYTES = P_STAGES * P_STAGE_BYTES;
+constexpr int P_GEMM_SMEM = P_TILE_BYTES + BAR_BYTES + 1024;
+
+template <int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                       const __grid_constant__ GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const uint32_t a_base = base;
+    const uint32_t b_base = base + P_STAGES * A_STAGE_BYTES;
+    const uint32_t bar_base = base + P_TILE_BYTES;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (P_STAGES + s); };
+    auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * P_STAGES + a); };
+    auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * P_STAGES + 2 + a); };
+    const uint32_t tmem_slot = bar_base + 8u * (2 * P_STAGES + 4);
+    volatile uint32_t* tmem_slot_ptr =
+        reinterpret_cast<volatile uint32_t*>(smem_raw + (base - raw) + P_TILE_BYTES + 8 * (2 * P_STAGES + 4));
+    __shared__ int s_failed;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();  // 0: leader (issues the MMAs), 1: peer
+    const int pair_id = blockIdx.x >> 1;
+    const int num_pairs = gridDim.x >> 1;
+    const int num_m = (p.M + 2 * BM - 1) / (2 * BM);  // tile-rows of 256
+    const int num_n = (p.N + BN - 1) / BN;
+    const int num_tiles = num_m * num_n;
+    const int num_kb = (p.K + BK - 1) / BK;
+    const int group_m = p.group_m > 0 ? p.group_m : 8;
+
+    if (threadIdx.x == 0) {
+        s_failed = 0;
+        for (int s = 0; s < P_STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(acc_full_bar(a), 1);
+            mbar_init(acc_empty_bar(a), 8);  // four epilogue warps in each CTA of the pair
+        }
+        fence_mbar_init();
+        tma_prefetch_desc(&tmap_a);
+        tma_prefetch_desc(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive();  // both CTAs' barriers exist before anyone signals across the pair
+    cluster_wait();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_ptr;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer (each CTA its own tiles)
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
+                const TileCoord tc = tile_coord(tile, num_m, num_n, group_m);
+                const int a_row = tc.m_idx * 2 * BM + static_cast<int>(rank) * BM;
+                const int b_row = tc.n_idx * BN + static_cast<int>(rank) * 128;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * P_STAGE_BYTES);  // both CTAs' bytes
+                    tma_load_2d_pair(a_base + stage * A_STAGE_BYTES, &tmap_a, kb * BK, a_row, leader_full);
+                    tma_load_2d_pair(b_base + stage * P_B_STAGE_BYTES, &tmap_b, kb * BK, b_row, leader_full);
+                    if (++stage == P_STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+            if (!ok) s_failed = 1;
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(2 * BM, BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
+                if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, p.status)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t a_desc = umma_desc_k_sw128(a_base + stage * A_STAGE_BYTES);
+                    const uint64_t b_desc = umma_desc_k_sw128(b_base + stage * P_B_STAGE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit_pair(empty_bar(stage));  // frees the stage in both CTAs
+                    if (++stage == P_STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit_pair(acc_full_bar(acc));  // accumulator ready in both CTAs
+                acc ^= 1;
+                if (acc == 0) acc_phase ^= 1u;
+            }
+            if (!ok) s_failed = 1;
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps 2..5 (both CTAs)
+        const int quarter = warp & 3;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
+            const TileCoord tc = tile_coord(tile, num_m, num_n, group_m);
+            if (!mbar_wait(acc_full_bar(acc), acc_phase, p.status)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const int row = tc.m_idx * 2 * BM + static_cast<int>(rank) * BM + quarter * 32 + lane;
+            const int n0 = tc.n_idx * BN;
+            const uint32_t trow = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
+            epilogue_tile<EPI>(p, trow, row, n0, tc.n_idx);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(acc), 0));  // the leader collects all 8
+            if constexpr (EPI == EPI_RESID_ADD_COMPARE) {
+                if (row < p.M && p.slot_first != nullptr) compare_row(p, row, n0, tc.n_idx, num_n);
+                __syncwarp();
+            }
+            acc ^= 1;
+            if (acc == 0) acc_phase ^= 1u;
+        }
+        if (!ok) s_failed = 1;
+    }
+
+    // ---------------------------------------------------------------- tail: neither CTA leaves while the other may
+    // still read its shared memory or signal its barriers
+    tc_fence_before();
+    __syncthreads();
+    if (s_failed) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {
+        }
+        __syncthreads();
+    }
+    cluster_arrive();
+    cluster_wait();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
+template <int EPI>
+cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int num_sms,
+                        cudaStream_t stream) {
+    const int num_tiles = ((p.M + 2 * BM - 1) / (2 * BM)) * ((p.N + BN - 1) / BN);
+    if (num_tiles <= 0) return cudaSuccess;
+    int pairs = num_sms / 2;
+    if (num_tiles < pairs) pairs = num_tiles;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs);
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = P_GEMM_SMEM;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_bf16_tcgen05_pair<EPI>, ta, tb, p);
+}
+
+template <int EPI>
+cudaError_t init_pair() {
+    return cudaFuncSetAttribute(gemm_bf16_tcgen05_pair<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_GEMM_SMEM);
+}
+
 template <int EPI>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int num_sms,
                        cudaStream_t stream) {
@@ -428,6 +642,12 @@ cudaError_t gemm_init() {
     if ((e = init_one<EPI_RESID_ADD>()) != cudaSuccess) return e;
     if ((e = init_one<EPI_SWIGLU>()) != cudaSuccess) return e;
     if ((e = init_one<EPI_RESID_ADD_COMPARE>()) != cudaSuccess) return e;
+    if ((e = init_pair<EPI_STORE_BF16>()) != cudaSuccess) return e;
+    if ((e = init_pair<EPI_STORE_F32>()) != cudaSuccess) return e;
+    if ((e = init_pair<EPI_QKV_ROPE>()) != cudaSuccess) return e;
+    if ((e = init_pair<EPI_RESID_ADD>()) != cudaSuccess) return e;
+    if ((e = init_pair<EPI_SWIGLU>()) != cudaSuccess) return e;
+    if ((e = init_pair<EPI_RESID_ADD_COMPARE>()) != cudaSuccess) return e;
     if (!g_encode) {
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -455,6 +675,17 @@ int make_tmap_bf16_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_
 
 cudaError_t launch_gemm(int epilogue, const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int num_sms,
                         cudaStream_t stream) {
+    if (p.pair) {  // tb must then be encoded with 128-row boxes (each CTA loads half of the B tile)
+        switch (epilogue) {
+            case EPI_STORE_BF16: return launch_pair<EPI_STORE_BF16>(ta, tb, p, num_sms, stream);
+            case EPI_STORE_F32: return launch_pair<EPI_STORE_F32>(ta, tb, p, num_sms, stream);
+            case EPI_QKV_ROPE: return launch_pair<EPI_QKV_ROPE>(ta, tb, p, num_sms, stream);
+            case EPI_RESID_ADD: return launch_pair<EPI_RESID_ADD>(ta, tb, p, num_sms, stream);
+            case EPI_SWIGLU: return launch_pair<EPI_SWIGLU>(ta, tb, p, num_sms, stream);
+            case EPI_RESID_ADD_COMPARE: return launch_pair<EPI_RESID_ADD_COMPARE>(ta, tb, p, num_sms, stream);
+            default: return cudaErrorInvalidValue;
+        }
+    }
     switch (epilogue) {
         case EPI_STORE_BF16: return launch_one<EPI_STORE_BF16>(ta, tb, p, num_sms, stream);
         case EPI_STORE_F32: return launch_one<EPI_STORE_F32>(ta, tb, p, num_sms, stream);

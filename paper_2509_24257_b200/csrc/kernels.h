@@ -27,7 +27,8 @@ struct GemmParams {
     int M, N, K;
     void* out;  // bf16 / fp32 matrix or the fp32 residual stream
     int ldo;    // leading dimension of out, elements
-    int group_m;  // tile-rows per band of the tile walk (0: default 16)
+    int group_m;  // tile-rows per band of the tile walk (0: default)
+    int pair;     // 1: CTA-pair kernel (256 x 256 tile over two SMs; B map encoded with 128-row boxes)
     // EPI_QKV_ROPE
     const float2* rope_cs;    // [position][head_dim/2] (cos, sin)
     const int* pos_of_token;  // [M]

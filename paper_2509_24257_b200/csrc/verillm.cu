@@ -15,6 +15,14 @@ namespace {
 
 typedef __nv_bfloat16 bf16;
 
+// Projections over more than 128 token rows run on CTA pairs (256 x 256 tiles over two SMs, each CTA loading
+// a 128-row half of the weight tile); smaller ones on single CTAs with 128 x 256 tiles.
+#ifdef VL_NO_PAIR
+inline int use_pair(int) { return 0; }
+#else
+inline int use_pair(int M) { return M > kGemmBM ? 1 : 0; }
+#endif
+
 #define CU_TRY(expr)                                  \
     do {                                              \
         cudaError_t _e = (expr);                      \
@@ -32,7 +40,8 @@ struct LayerDev {
     bf16 *wo = nullptr;    // [d][H dh]
     bf16 *wgu = nullptr;   // [2 F][d]: blocks of 128 gate rows followed by the 128 matching up rows
     bf16 *wd = nullptr;    // [d][F]
-    CUtensorMap t_wqkv, t_wo, t_wgu, t_wd;
+    CUtensorMap t_wqkv, t_wo, t_wgu, t_wd;          // boxes of 256 weight rows (single-CTA tiles)
+    CUtensorMap t_wqkv_h, t_wo_h, t_wgu_h, t_wd_h;  // boxes of 128 weight rows (one half per CTA of a pair)
 };
 
 struct DecodeState {
@@ -192,6 +201,7 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
     std::memset(&p, 0, sizeof(p));
     p.status = status;
     p.M = r.M;
+    p.pair = use_pair(r.M);
     // Activations of the K = d_model projections (M x d bf16) stay L2-resident when the band spans every
     // tile-row, so each weight tile is fetched from HBM once; the down projection streams a wider A.
     const int num_m = (r.M + kGemmBM - 1) / kGemmBM;
@@ -199,13 +209,16 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
 #define VL_BAND_L2_BYTES 0u
 #endif
     const bool a_fits_l2 = static_cast<size_t>(r.M) * c.d_model * 2 <= VL_BAND_L2_BYTES;  // measured: bands of 16 win
-    const int band_d = a_fits_l2 ? num_m : 16;
+    #ifndef VL_PAIR_BAND
+#define VL_PAIR_BAND 8
+#endif
+    const int band_d = a_fits_l2 ? num_m : (p.pair ? VL_PAIR_BAND : 16);
 
     CU_TRY(launch_rmsnorm(m->resid, w.attn_norm, m->xn, r.M, c.d_model, c.rms_eps, st));
     prof_mark(m, VERILLM_PROF_RMSNORM, st);
     p.N = m->n_qkv; p.K = c.d_model; p.out = m->qkv; p.ldo = m->n_qkv; p.group_m = band_d;
     p.rope_cs = m->rope_cs; p.pos_of_token = m->pos_of_token; p.head_dim = c.head_dim; p.rope_cols = m->d_q + m->d_kv;
-    CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, w.t_wqkv, p, m->num_sms, st));
+    CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, p.pair ? w.t_wqkv_h : w.t_wqkv, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_QKV, st);
 #ifdef VL_ATTN_LEGACY
     CU_TRY(launch_attention(m->qkv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads, c.head_dim, m->attn, st));
@@ -215,23 +228,23 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
 #endif
     prof_mark(m, VERILLM_PROF_ATTENTION, st);
     p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
-    p.group_m = static_cast<size_t>(r.M) * m->d_q * 2 <= VL_BAND_L2_BYTES ? num_m : 16;
-    CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_attn, w.t_wo, p, m->num_sms, st));
+    p.group_m = band_d;
+    CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_attn, p.pair ? w.t_wo_h : w.t_wo, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_O, st);
     CU_TRY(launch_rmsnorm(m->resid, w.ffn_norm, m->xn, r.M, c.d_model, c.rms_eps, st));
     prof_mark(m, VERILLM_PROF_RMSNORM, st);
     p.N = 2 * c.d_ffn; p.K = c.d_model; p.out = m->mid; p.ldo = c.d_ffn; p.group_m = band_d;
-    CU_TRY(launch_gemm(EPI_SWIGLU, m->t_xn, w.t_wgu, p, m->num_sms, st));
+    CU_TRY(launch_gemm(EPI_SWIGLU, m->t_xn, p.pair ? w.t_wgu_h : w.t_wgu, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_GATE_UP, st);
     p.N = c.d_model; p.K = c.d_ffn; p.out = m->resid; p.ldo = c.d_model;
-    p.group_m = static_cast<size_t>(r.M) * c.d_ffn * 2 <= VL_BAND_L2_BYTES ? num_m : 16;
+    p.group_m = band_d;
     if (r.cmp_layer) {
         p.slot_first = r.cmp_layer->slot_first; p.slot_next = r.cmp_layer->slot_next; p.n_check = r.cmp_layer->n_check;
         p.committed = r.cmp_layer->committed; p.partials = r.cmp_layer->partials; p.hidden_out = r.cmp_layer->hidden_out;
         p.cmp = r.cmp_layer->cmp;
-        CU_TRY(launch_gemm(EPI_RESID_ADD_COMPARE, m->t_mid, w.t_wd, p, m->num_sms, st));
+        CU_TRY(launch_gemm(EPI_RESID_ADD_COMPARE, m->t_mid, p.pair ? w.t_wd_h : w.t_wd, p, m->num_sms, st));
     } else {
-        CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_mid, w.t_wd, p, m->num_sms, st));
+        CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_mid, p.pair ? w.t_wd_h : w.t_wd, p, m->num_sms, st));
     }
     prof_mark(m, VERILLM_PROF_GEMM_DOWN, st);
     *launches += 7;
@@ -453,10 +466,13 @@ int verillm_load_weights(const verillm_config* cfg, const verillm_weights* weigh
     ok = ok && make_tmap_bf16_2d(&m->t_qkv_q, m->qkv, T, m->n_qkv, m->n_qkv, 128) == 0;
     ok = ok && make_tmap_bf16_2d(&m->t_qkv_kv, m->qkv, T, m->n_qkv, m->n_qkv, 64) == 0;
     for (LayerDev& L : m->layers) {
-        ok = ok && make_tmap_bf16_2d(&L.t_wqkv, L.wqkv, m->n_qkv, d, d, kGemmBN) == 0;
-        ok = ok && make_tmap_bf16_2d(&L.t_wo, L.wo, d, m->d_q, m->d_q, kGemmBN) == 0;
-        ok = ok && make_tmap_bf16_2d(&L.t_wgu, L.wgu, 2 * static_cast<uint64_t>(c.d_ffn), d, d, kGemmBN) == 0;
-        ok = ok && make_tmap_bf16_2d(&L.t_wd, L.wd, d, c.d_ffn, c.d_ffn, kGemmBN) == 0;
+        for (int half = 0; half < 2; ++half) {
+            const uint32_t box = half ? 128 : kGemmBN;
+            ok = ok && make_tmap_bf16_2d(half ? &L.t_wqkv_h : &L.t_wqkv, L.wqkv, m->n_qkv, d, d, box) == 0;
+            ok = ok && make_tmap_bf16_2d(half ? &L.t_wo_h : &L.t_wo, L.wo, d, m->d_q, m->d_q, box) == 0;
+            ok = ok && make_tmap_bf16_2d(half ? &L.t_wgu_h : &L.t_wgu, L.wgu, 2 * static_cast<uint64_t>(c.d_ffn), d, d, box) == 0;
+            ok = ok && make_tmap_bf16_2d(half ? &L.t_wd_h : &L.t_wd, L.wd, d, c.d_ffn, c.d_ffn, box) == 0;
+        }
     }
     if (!ok) {
         verillm_free(m);
@@ -770,10 +786,10 @@ int verillm_op_gemm(const void* a, const void* b, void* cmat, int32_t M, int32_t
     CU_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     CUtensorMap ta, tb;
     if (make_tmap_bf16_2d(&ta, a, M, K, K, kGemmBM) != 0) return VERILLM_E_CUDA;
-    if (make_tmap_bf16_2d(&tb, b, N, K, K, kGemmBN) != 0) return VERILLM_E_CUDA;
+    if (make_tmap_bf16_2d(&tb, b, N, K, K, use_pair(M) ? 128 : kGemmBN) != 0) return VERILLM_E_CUDA;
     GemmParams p;
     std::memset(&p, 0, sizeof(p));
-    p.M = M; p.N = N; p.K = K; p.out = cmat; p.ldo = N; p.status = status;
+    p.M = M; p.N = N; p.K = K; p.out = cmat; p.ldo = N; p.status = status; p.pair = use_pair(M);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (status) CU_TRY(cudaMemsetAsync(status, 0, sizeof(int), st));
     CU_TRY(launch_gemm(out_f32 ? EPI_STORE_F32 : EPI_STORE_BF16, ta, tb, p, sms, st));
