@@ -191,18 +191,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             tmem_ld32(s_addr, v0);
             tmem_ld32(s_addr + 32, v1);
             tmem_ld_wait();
+            // raw scores: mask the future on the diagonal tiles only, then one maximum per row
+            if (need_mask) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    if (key0 + i > row) v0[i] = 0xFF800000u;       // -inf
+                    if (key0 + 32 + i > row) v1[i] = 0xFF800000u;
+                }
+            }
             float mx = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                float x0 = __uint_as_float(v0[i]) * scale_log2, x1 = __uint_as_float(v1[i]) * scale_log2;
-                if (need_mask) {
-                    if (key0 + i > row) x0 = -INFINITY;
-                    if (key0 + 32 + i > row) x1 = -INFINITY;
-                }
-                v0[i] = __float_as_uint(x0);
-                v1[i] = __float_as_uint(x1);
-                mx = fmaxf(mx, fmaxf(x0, x1));
-            }
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(v0[i]), __uint_as_float(v1[i])));
+            mx *= scale_log2;  // the scale is positive: max commutes with it
             if (j == 0) {
                 m_ref = mx;  // tile 0 holds key 0 <= row: finite
             } else {
@@ -231,8 +231,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             uint32_t pk[32];
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-                const float a0 = ex2(__uint_as_float(v0[2 * i]) - m_ref), a1 = ex2(__uint_as_float(v0[2 * i + 1]) - m_ref);
-                const float b0 = ex2(__uint_as_float(v1[2 * i]) - m_ref), b1 = ex2(__uint_as_float(v1[2 * i + 1]) - m_ref);
+                const float a0 = ex2(fmaf(__uint_as_float(v0[2 * i]), scale_log2, -m_ref));
+                const float a1 = ex2(fmaf(__uint_as_float(v0[2 * i + 1]), scale_log2, -m_ref));
+                const float b0 = ex2(fmaf(__uint_as_float(v1[2 * i]), scale_log2, -m_ref));
+                const float b1 = ex2(fmaf(__uint_as_float(v1[2 * i + 1]), scale_log2, -m_ref));
                 rs += (a0 + a1) + (b0 + b1);
                 pk[i] = pack_bf16(a0, a1);
                 pk[16 + i] = pack_bf16(b0, b1);

@@ -210,7 +210,7 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
 #endif
     const bool a_fits_l2 = static_cast<size_t>(r.M) * c.d_model * 2 <= VL_BAND_L2_BYTES;  // measured: bands of 16 win
     #ifndef VL_PAIR_BAND
-#define VL_PAIR_BAND 8
+#define VL_PAIR_BAND 16
 #endif
     const int band_d = a_fits_l2 ? num_m : (p.pair ? VL_PAIR_BAND : 16);
 
