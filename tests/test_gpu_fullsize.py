@@ -83,3 +83,42 @@ def test_llama8b_full_depth_sampled_positions_and_honest_trace():
     assert np.array_equal(rep2["hidden"], g["hidden"][:, sub])
     assert np.array_equal(rep2["stats"], g["stats"][sub])
     model.close()
+
+
+def _sampled_parity(wl, sampled, bad_slot, bad_layer, oracle_device=DEV):
+    """Runs the whole batch on the GPU and the oracle on the sampled (sequence, position) pairs only."""
+    tokens = synth.token_streams(wl)
+    cs = np.array([s for s, _ in sampled], np.int32)
+    cp = np.array([p for _, p in sampled], np.int32)
+    model = H.gpu_model(wl, len(cs))
+    om = H.oracle_model_streamed(wl, np.concatenate([tokens[s][: p + 1] for s, p in sampled]), oracle_device)
+    zeros = np.zeros((wl.shape.n_layers, len(cs), wl.shape.d_model))
+    pre = vo.verify_prefill(om, list(tokens), zeros, cs, cp, vo.Tol(), "bf16", prefix_only=True)
+    honest = vo.round_to_bf16(pre.hidden)
+    tampered = synth.add_state_noise(honest, [bad_slot], [bad_layer], 10 * 5e-2, synth.tamper_rng(wl))
+    comm = synth.to_commit_dtype(tampered, "bf16")
+    flat = torch.from_numpy(tokens.reshape(-1)).to(DEV)
+    g = model.verify_prefill(flat, synth.cu_seqlens(wl), comm.to(DEV), cs, cp, want_hidden=True).cpu()
+    model.close()
+    stats_o = np.transpose(vo.compare_stats(pre.hidden, comm.to(torch.float64).numpy(), "bf16", vo.Tol()), (1, 0, 2))
+    pos_ok_o, first_bad_o, seq_ok_o, _ = vo.verdict(stats_o, cs, wl.batch, vo.Tol())
+    assert g["status"] == 0
+    rel = H.rel_l2(g["hidden"], pre.hidden)
+    assert rel.max() <= 2e-2, rel.max()
+    assert np.array_equal(g["pos_ok"], pos_ok_o) and np.array_equal(g["first_bad_layer"], first_bad_o)
+    assert np.array_equal(g["seq_ok"], seq_ok_o)
+    assert g["pos_ok"][bad_slot] == 0 and g["pos_ok"].sum() == len(cs) - 1 and g["first_bad_layer"][bad_slot] == bad_layer
+    assert np.all(np.abs(g["stats"][..., REL] - stats_o[..., REL]) <= 2.4e-2)
+
+
+def test_long_context_8b_width_sparse_checks():
+    """2 sequences of 4096 tokens at the 8B widths (two layers): 64 key tiles per query tile in attention, and
+    checks as sparse as one per thousand rows, among them the very last position of a sequence."""
+    wl = synth.WORKLOADS["llama8b_long"].with_layers(2)
+    _sampled_parity(wl, [(0, 5), (0, 700), (1, 2048), (1, 4095)], bad_slot=1, bad_layer=1)
+
+
+def test_llama70b_width_single_layer():
+    """Llama-3-70B widths (d 8192, 64/8 heads, FFN 28672), one layer, the configured 1 x 2048 batch."""
+    wl = synth.WORKLOADS["llama70b"].with_layers(1)
+    _sampled_parity(wl, [(0, 0), (0, 63), (0, 129), (0, 300)], bad_slot=2, bad_layer=0)
