@@ -30,6 +30,7 @@ sys.path.insert(0, ROOT)
 METRIC, UNIT = "verified_tokens_per_sec", "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 TOL_REL_L2 = 5e-2
+GATE_UP_DRAM_BYTES_8B = 791.4e6 + 226.6e6  # measured, per launch, M = 8192 tokens at the 8B widths
 
 
 def measured_peaks():
@@ -325,8 +326,11 @@ def run_ours(args, wl):
     dom = "gemm_gate_up_swiglu"
     achieved = flops_per_launch[dom] / (acc[dom][0] / acc[dom][1] * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
+    # DRAM bytes of one launch of that kernel (dram__bytes_read.sum + dram__bytes_write.sum from the ncu capture
+    # summarised in profiles/layer_kernels_llama8b_ncu_full.md); only valid for the shape it was taken on
+    traffic = GATE_UP_DRAM_BYTES_8B if (s.d_model, s.d_ffn, M) == (4096, 14336, 8192) else None
     roofline = {"bound": "tensor", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "TFLOP/s",
-                "frac": round(achieved / peak, 4), "traffic": None,
+                "frac": round(achieved / peak, 4), "traffic": traffic,
                 "peak_kind": f"bf16 sustained, of {peaks_kind}", "kernels": kernels}
 
     if rank == 0:
