@@ -103,7 +103,6 @@ int ensure_init() {
     CU_TRY(cudaGetDeviceProperties(&prop, dev));
     if (prop.major != 10) return VERILLM_E_ARCH;
     CU_TRY(gemm_init());
-    CU_TRY(attention_init());
     CU_TRY(attention_tc_init());
     done[dev] = true;
     return VERILLM_OK;
@@ -220,12 +219,8 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
     p.rope_cs = m->rope_cs; p.pos_of_token = m->pos_of_token; p.head_dim = c.head_dim; p.rope_cols = m->d_q + m->d_kv;
     CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, p.pair ? w.t_wqkv_h : w.t_wqkv, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_QKV, st);
-#ifdef VL_ATTN_LEGACY
-    CU_TRY(launch_attention(m->qkv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads, c.head_dim, m->attn, st));
-#else
     CU_TRY(launch_attention_tc(m->t_qkv_q, m->t_qkv_kv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads,
                                c.head_dim, m->attn, status, st));
-#endif
     prof_mark(m, VERILLM_PROF_ATTENTION, st);
     p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
     p.group_m = band_d;
@@ -810,17 +805,12 @@ int verillm_op_attention(const void* qkv, const int32_t* cu_seqlens, int32_t bat
         return VERILLM_E_SHAPE;
     int rc = ensure_init();
     if (rc) return rc;
-#ifdef VL_ATTN_LEGACY
-    CU_TRY(launch_attention(qkv, cu_seqlens, batch, max_seqlen, n_heads, n_kv_heads, head_dim, out,
-                            reinterpret_cast<cudaStream_t>(cuda_stream)));
-#else
     const int n_qkv = (n_heads + 2 * n_kv_heads) * head_dim;
     CUtensorMap tq, tkv;
     if (make_tmap_bf16_2d(&tq, qkv, M, n_qkv, n_qkv, 128) != 0) return VERILLM_E_CUDA;
     if (make_tmap_bf16_2d(&tkv, qkv, M, n_qkv, n_qkv, 64) != 0) return VERILLM_E_CUDA;
     CU_TRY(launch_attention_tc(tq, tkv, cu_seqlens, batch, max_seqlen, n_heads, n_kv_heads, head_dim, out, nullptr,
                                reinterpret_cast<cudaStream_t>(cuda_stream)));
-#endif
     return VERILLM_OK;
 }
 
