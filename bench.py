@@ -333,6 +333,26 @@ def run_ours(args, wl):
                 "frac": round(achieved / peak, 4), "traffic": traffic,
                 "peak_kind": f"bf16 sustained, of {peaks_kind}", "kernels": kernels}
 
+    # ---- tail token check (next row of the scope table): final norm + output head + arg-max on the checked rows;
+    # it streams the [vocab][d_model] head once, so it is reported against the measured copy bandwidth
+    from paper_2509_24257_b200 import synth as _synth
+    model.load_lm_head(_synth.lm_head_weights(wl, device))
+    last_hidden = torch.randn(len(cs), s.d_model, device=device)
+    claimed = np.zeros(len(cs), dtype=np.int32)
+    for _ in range(3):
+        model.token_match(last_hidden, claimed, stream)
+    t0e, t1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0e.record(stream)
+    for _ in range(20):
+        model.token_match(last_hidden, claimed, stream)
+    t1e.record(stream)
+    torch.cuda.synchronize()
+    tm_ms = t0e.elapsed_time(t1e) / 20
+    tm_bytes = s.vocab * s.d_model * 2 + len(cs) * s.d_model * 6
+    token_match = {"rows": int(len(cs)), "ms": round(tm_ms, 4), "bound": "hbm",
+                   "achieved_gbs": round(tm_bytes / (tm_ms * 1e-3) / 1e9, 1), "peak_gbs": peaks["hbm_gbs"],
+                   "frac": round(tm_bytes / (tm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
+
     if rank == 0:
         run, desc = oracle_sample(wl, 12.0, str(device)) if args.gpus == 1 else (None, None)
         cpu_baseline = None
@@ -359,7 +379,8 @@ def run_ours(args, wl):
                          "status": res["status"]},
             "clocks": clocks, "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                                      "d2h_bytes_per_step": int(d2h)},
-            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "gpu_launches": int(launches), "roofline": roofline, "token_match": token_match,
+            "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))
     model.close()

@@ -170,6 +170,22 @@ int verillm_decode_commit(verillm_model *model, const int32_t *tokens, const int
                           int32_t n_prefill, const int32_t *check_seq, const int32_t *check_pos, int32_t n_check,
                           void *committed_out, int32_t commit_dtype, int32_t *status, void *cuda_stream);
 
+/* Tail token check ("TokenMatch(argmax f_LM(S_{L+1}), y) = 1"; token-state cross-check of the forged-output
+ * analysis): the last-layer states at the checked positions go through the final RMSNorm and the output
+ * head, and the arg-max token of each row is compared with the token the prover claims to have emitted there.
+ *  verillm_load_lm_head: output head [vocab][d_model] bf16 (HOST or DEVICE per on_device); the first call also
+ *                        allocates the scratch of the check inside the handle.  vocab % 32 == 0 (else E_SHAPE).
+ *  last_hidden  DEVICE float32 [n_check][d_model]: e.g. the last layer of verify_prefill's hidden_out
+ *  claimed      HOST int32 [n_check]: the next token the prover reported for that position
+ *  argmax_out   DEVICE int32 [n_check]; match_out DEVICE uint8 [n_check] (1 = equal);
+ *  margin_out   DEVICE float [n_check]: best logit minus runner-up (a small margin marks a row whose arg-max
+ *               rounding noise may flip).  Ties resolve to the lowest token id.
+ * Allocates nothing per call.  Errors: E_INVAL (also when no output head was loaded), E_SHAPE (n_check >
+ * max_checks). */
+int verillm_load_lm_head(verillm_model *model, const void *lm_head, int32_t on_device);
+int verillm_token_match(verillm_model *model, const float *last_hidden, const int32_t *claimed, int32_t n_check,
+                        int32_t *argmax_out, uint8_t *match_out, float *margin_out, void *cuda_stream);
+
 /* Comparison and verdict alone, on states the caller already holds (Delta = S_hat - S, phi, Psi, b):
  *  hidden    DEVICE float32 [n_layers][n_check][d_model]
  *  committed DEVICE [n_layers][n_check][d_model] in commit_dtype

@@ -404,6 +404,19 @@ def verdict(stats: np.ndarray, check_seq: np.ndarray, batch: int, tol: Tol):
     return pos_ok.astype(np.uint8), first_bad, seq_ok, seq_score
 
 
+def token_match(m: Model, last_hidden: np.ndarray, lm_head: np.ndarray, claimed: np.ndarray):
+    """Tail token check: TokenMatch(argmax f_LM(S_{L+1}), y) with f_LM = output head after the final RMSNorm.
+
+    last_hidden [n, d_model] (states after the last block), lm_head [vocab, d_model] (float or bf16 bits),
+    claimed [n].  Returns (argmax [n], match [n] uint8, margin [n] = best logit - runner-up).  np.argmax
+    takes the lowest index among equal maxima."""
+    logits = rmsnorm(np.asarray(last_hidden, dtype=np.float64), m.final_norm, m.rms_eps) @ as_f64(lm_head).T
+    arg = np.argmax(logits, axis=-1)
+    top2 = np.partition(logits, -2, axis=-1)[:, -2:]
+    margin = top2[:, 1] - top2[:, 0]
+    return arg.astype(np.int32), (arg == np.asarray(claimed)).astype(np.uint8), margin
+
+
 def verify_prefill(
     m: Model, seqs: Sequence[np.ndarray], committed: np.ndarray, check_seq: np.ndarray,
     check_pos: np.ndarray, tol: Tol, commit_dtype: str = "bf16", prefix_only: bool = False,

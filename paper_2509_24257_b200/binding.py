@@ -30,6 +30,7 @@ EXPORTS = (
     "verillm_verify_prefill", "verillm_decode_commit", "verillm_compare", "verillm_compare_noalloc", "verillm_op_gemm",
     "verillm_op_rmsnorm", "verillm_op_attention", "verillm_free", "verillm_strerror",
     "verillm_last_launch_count", "verillm_profile_enable", "verillm_profile_read",
+    "verillm_load_lm_head", "verillm_token_match",
 )
 PROF_CLASSES = ("setup", "rmsnorm", "gemm_qkv_rope", "attention", "gemm_o_resid", "gemm_gate_up_swiglu",
                 "gemm_down_resid_compare", "verdict")
@@ -108,6 +109,10 @@ def lib() -> C.CDLL:
         ]
         L.verillm_compare_noalloc.argtypes = L.verillm_compare.argtypes
         L.verillm_compare_noalloc.restype = C.c_int
+        L.verillm_load_lm_head.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
+        L.verillm_load_lm_head.restype = C.c_int
+        L.verillm_token_match.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.verillm_token_match.restype = C.c_int
         L.verillm_op_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.verillm_op_rmsnorm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p]
         L.verillm_op_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
@@ -273,6 +278,26 @@ class Model:
         if int(status.item()) != 0:
             raise RuntimeError(f"verillm_decode_commit: device status {int(status.item())}")
         return out[:, :n_check]
+
+    def load_lm_head(self, lm_head: torch.Tensor) -> None:
+        if lm_head.dtype != torch.bfloat16 or not lm_head.is_contiguous():
+            raise ValueError("the output head must be contiguous bf16")
+        with torch.cuda.device(self.device):
+            _check(lib().verillm_load_lm_head(self._h, lm_head.data_ptr(), int(lm_head.is_cuda)), "verillm_load_lm_head")
+
+    def token_match(self, last_hidden: torch.Tensor, claimed: Sequence[int], stream: Optional[torch.cuda.Stream] = None):
+        """last_hidden: float32 device [n_check][d_model].  Returns device tensors (argmax int32, match uint8, margin f32)."""
+        cl = _i32(claimed)
+        n = int(cl.shape[0])
+        if last_hidden.dtype != torch.float32 or not last_hidden.is_contiguous() or last_hidden.shape[0] != n:
+            raise ValueError("last_hidden must be contiguous float32 [n_check][d_model]")
+        arg = torch.empty(n, dtype=torch.int32, device=self.device)
+        match = torch.empty(n, dtype=torch.uint8, device=self.device)
+        margin = torch.empty(n, dtype=torch.float32, device=self.device)
+        with torch.cuda.device(self.device):
+            _check(lib().verillm_token_match(self._h, last_hidden.data_ptr(), cl.ctypes.data, n, arg.data_ptr(),
+                                             match.data_ptr(), margin.data_ptr(), _stream_ptr(stream)), "verillm_token_match")
+        return arg, match, margin
 
     def profile_enable(self, on: bool = True) -> None:
         with torch.cuda.device(self.device):

@@ -236,6 +236,48 @@ __global__ void seq_verdict_kernel(const float* __restrict__ stats, const uint8_
     }
 }
 
+// ------------------------------------------------------------------ tail token check
+// One warp per row: lanes take column tiles in a strided order, records are merged with "larger value, then
+// lower column" so the result does not depend on the merge order; match = (argmax == claimed token).
+struct Top2 {
+    float best, second;
+    int col;
+};
+__device__ __forceinline__ Top2 top2_merge(const Top2& a, const Top2& b) {
+    const bool a_wins = a.best > b.best || (a.best == b.best && a.col < b.col);
+    Top2 r;
+    r.best = a_wins ? a.best : b.best;
+    r.col = a_wins ? a.col : b.col;
+    r.second = fmaxf(fmaxf(a.second, b.second), a_wins ? b.best : a.best);
+    return r;
+}
+__global__ void argmax_reduce_kernel(const float4* __restrict__ records, int rows, int n_tiles,
+                                     const int* __restrict__ claimed, int* __restrict__ argmax_out,
+                                     uint8_t* __restrict__ match_out, float* __restrict__ margin_out) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    Top2 t = {-INFINITY, -INFINITY, 0x7FFFFFFF};
+    for (int i = lane; i < n_tiles; i += 32) {
+        const float4 r = records[static_cast<size_t>(row) * n_tiles + i];
+        const Top2 u = {r.x, r.z, __float_as_int(r.y)};
+        t = top2_merge(t, u);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Top2 u;
+        u.best = __shfl_xor_sync(0xFFFFFFFFu, t.best, o);
+        u.second = __shfl_xor_sync(0xFFFFFFFFu, t.second, o);
+        u.col = __shfl_xor_sync(0xFFFFFFFFu, t.col, o);
+        t = top2_merge(t, u);
+    }
+    if (lane == 0) {
+        argmax_out[row] = t.col;
+        match_out[row] = (t.col == claimed[row]) ? 1 : 0;
+        margin_out[row] = t.best - t.second;
+    }
+}
+
 // ------------------------------------------------------------------ decode-side kernels
 // out[r][n] (+)= sum_k x[r][k] * w[n][k] for up to 8 rows: one warp per output column streams the
 // weight row once (16-byte loads) and keeps one accumulator per row.
@@ -461,6 +503,14 @@ cudaError_t launch_seq_verdict(const float* stats, const uint8_t* pos_ok, const 
     if (batch <= 0) return cudaSuccess;
     seq_verdict_kernel<<<(batch + 3) / 4, 128, 0, s>>>(stats, pos_ok, seq_of_slot, n_check, n_layers, batch, seq_ok,
                                                         seq_score);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_argmax_reduce(const float* records, int rows, int n_tiles, const int* claimed, int* argmax_out,
+                                 uint8_t* match_out, float* margin_out, cudaStream_t s) {
+    if (rows <= 0) return cudaSuccess;
+    argmax_reduce_kernel<<<(rows + 3) / 4, 128, 0, s>>>(reinterpret_cast<const float4*>(records), rows, n_tiles, claimed,
+                                                       argmax_out, match_out, margin_out);
     return cudaGetLastError();
 }
 

@@ -75,7 +75,34 @@ template <int EPI>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t trow, int row, int n0, int n_idx) {
     const bool row_ok = row < p.M;
 
-    if constexpr (EPI == EPI_STORE_BF16 || EPI == EPI_STORE_F32) {
+    if constexpr (EPI == EPI_ARGMAX) {
+        // largest and second largest accumulator of the row inside this column tile (first column wins ties)
+        float best = -INFINITY, second = -INFINITY;
+        int best_col = n0;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            const int col = n0 + c * 32;
+            if (col >= p.N) break;
+            float v[32];
+            load_acc(trow + c * 32, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float x = v[i];
+                if (x > best) {
+                    second = best;
+                    best = x;
+                    best_col = col + i;
+                } else {
+                    second = fmaxf(second, x);
+                }
+            }
+        }
+        if (row_ok && n0 < p.N) {
+            const int n_tiles = (p.N + BN - 1) / BN;
+            float4* rec = reinterpret_cast<float4*>(p.out) + static_cast<size_t>(row) * n_tiles + n_idx;
+            *rec = make_float4(best, __int_as_float(best_col), second, 0.f);
+        }
+    } else if constexpr (EPI == EPI_STORE_BF16 || EPI == EPI_STORE_F32) {
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
             const int col = n0 + c * 32;
@@ -648,6 +675,8 @@ cudaError_t gemm_init() {
     if ((e = init_pair<EPI_RESID_ADD>()) != cudaSuccess) return e;
     if ((e = init_pair<EPI_SWIGLU>()) != cudaSuccess) return e;
     if ((e = init_pair<EPI_RESID_ADD_COMPARE>()) != cudaSuccess) return e;
+    if ((e = init_one<EPI_ARGMAX>()) != cudaSuccess) return e;
+    if ((e = init_pair<EPI_ARGMAX>()) != cudaSuccess) return e;
     if (!g_encode) {
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -683,6 +712,7 @@ cudaError_t launch_gemm(int epilogue, const CUtensorMap& ta, const CUtensorMap& 
             case EPI_RESID_ADD: return launch_pair<EPI_RESID_ADD>(ta, tb, p, num_sms, stream);
             case EPI_SWIGLU: return launch_pair<EPI_SWIGLU>(ta, tb, p, num_sms, stream);
             case EPI_RESID_ADD_COMPARE: return launch_pair<EPI_RESID_ADD_COMPARE>(ta, tb, p, num_sms, stream);
+            case EPI_ARGMAX: return launch_pair<EPI_ARGMAX>(ta, tb, p, num_sms, stream);
             default: return cudaErrorInvalidValue;
         }
     }
@@ -693,6 +723,7 @@ cudaError_t launch_gemm(int epilogue, const CUtensorMap& ta, const CUtensorMap& 
         case EPI_RESID_ADD: return launch_one<EPI_RESID_ADD>(ta, tb, p, num_sms, stream);
         case EPI_SWIGLU: return launch_one<EPI_SWIGLU>(ta, tb, p, num_sms, stream);
         case EPI_RESID_ADD_COMPARE: return launch_one<EPI_RESID_ADD_COMPARE>(ta, tb, p, num_sms, stream);
+        case EPI_ARGMAX: return launch_one<EPI_ARGMAX>(ta, tb, p, num_sms, stream);
         default: return cudaErrorInvalidValue;
     }
 }

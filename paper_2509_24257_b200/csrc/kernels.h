@@ -16,7 +16,8 @@ enum GemmEpilogue {
     EPI_QKV_ROPE = 2,        // C bf16, rotary embedding on the q and k head columns
     EPI_RESID_ADD = 3,       // resid fp32 += acc (in place)
     EPI_SWIGLU = 4,          // tile holds 128 gate columns then 128 up columns: out bf16 = silu(g) * u
-    EPI_RESID_ADD_COMPARE = 5  // resid += acc, then gather-and-compare on the checked rows
+    EPI_RESID_ADD_COMPARE = 5,  // resid += acc, then gather-and-compare on the checked rows
+    EPI_ARGMAX = 6              // no matrix output: per row and column tile (best value, its column, runner-up)
 };
 
 constexpr int kGemmBM = 128;
@@ -34,6 +35,7 @@ struct GemmParams {
     const int* pos_of_token;  // [M]
     int head_dim;
     int rope_cols;  // columns [0, rope_cols) hold heads that are rotated (q and k); the rest (v) are not
+    // EPI_ARGMAX: `out` is float [M][n_tiles][4] = (best, column as int bits, runner-up, unused)
     // EPI_RESID_ADD_COMPARE (slabs of the current layer)
     const int* slot_first;  // [M] first check slot of a token row, -1 if none
     const int* slot_next;   // [n_check] next slot on the same row, -1 terminates
@@ -80,6 +82,11 @@ cudaError_t launch_verdict(const float* partials, int n_layers, int n_check, int
                            cudaStream_t stream);
 cudaError_t launch_seq_verdict(const float* stats, const uint8_t* pos_ok, const int* seq_of_slot, int n_check,
                                int n_layers, int batch, uint8_t* seq_ok, float* seq_score, cudaStream_t stream);
+
+// Tail token check: reduces the per-tile argmax records of the output-head product [rows][n_tiles][4] (fixed order,
+// lowest column wins ties), compares with the claimed tokens.
+cudaError_t launch_argmax_reduce(const float* records, int rows, int n_tiles, const int* claimed, int* argmax_out,
+                                 uint8_t* match_out, float* margin_out, cudaStream_t stream);
 
 // ------------------------------------------------------------------ decode (prover side)
 // out[rows][n] (fp32) = x[rows][k] (bf16) * w[n][k]^T, rows <= 8 per launch group; optional in-place add.

@@ -78,6 +78,12 @@ struct verillm_model {
     float2* rope_cs = nullptr;
     CUtensorMap t_xn, t_attn, t_mid;
     CUtensorMap t_qkv_q, t_qkv_kv;  // attention operands: boxes of 128 query rows / 64 key rows
+    // tail token check (allocated by verillm_load_lm_head)
+    bf16 *lm_head = nullptr, *tm_y = nullptr;
+    float* tm_rec = nullptr;
+    int* tm_claimed = nullptr;
+    int n_tiles_v = 0;
+    CUtensorMap t_lm, t_lm_h, t_tm_y;
     DecodeState dec;
     Profile prof;
     int last_launches = 0;
@@ -304,6 +310,7 @@ void verillm_free(verillm_model* m) {
     cudaFree(m->pos_of_token); cudaFree(m->seq_of_token); cudaFree(m->slot_first); cudaFree(m->slot_next);
     cudaFree(m->tok_of_slot); cudaFree(m->seq_of_slot); cudaFree(m->cu_dev); cudaFree(m->status);
     cudaFree(m->partials); cudaFree(m->rope_cs);
+    cudaFree(m->lm_head); cudaFree(m->tm_y); cudaFree(m->tm_rec); cudaFree(m->tm_claimed);
     DecodeState& d = m->dec;
     cudaFree(d.kv_cache); cudaFree(d.hidden_tmp); cudaFree(d.resid); cudaFree(d.qkv); cudaFree(d.gu);
     cudaFree(d.xn); cudaFree(d.q); cudaFree(d.attn); cudaFree(d.mid); cudaFree(d.ints);
@@ -616,6 +623,48 @@ int verillm_compare_noalloc(const float* hidden, const void* committed, int32_t 
     CU_TRY(launch_verdict(partials, n_layers, n_check, 1, d_model, tol_dev(*tol), rep->status, rep->stats, rep->pos_ok,
                           rep->first_bad_layer, st));
     CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, seq_dev, n_check, n_layers, batch, rep->seq_ok, rep->seq_score, st));
+    return VERILLM_OK;
+}
+
+int verillm_load_lm_head(verillm_model* m, const void* lm_head, int32_t on_device) {
+    if (!m || !lm_head) return VERILLM_E_INVAL;
+    const verillm_config& c = m->cfg;
+    if (c.vocab % 32 != 0) return VERILLM_E_SHAPE;
+    const size_t d = c.d_model, NC = std::max(c.max_checks, 1);
+    int rc;
+    if (!m->lm_head) {
+        m->n_tiles_v = (c.vocab + kGemmBN - 1) / kGemmBN;
+        if ((rc = dev_alloc(&m->lm_head, static_cast<size_t>(c.vocab) * d))) return rc;
+        if ((rc = dev_alloc(&m->tm_y, NC * d))) return rc;
+        if ((rc = dev_alloc(&m->tm_rec, NC * m->n_tiles_v * 4))) return rc;
+        if ((rc = dev_alloc(&m->tm_claimed, NC))) return rc;
+        CU_TRY(cudaMemset(m->tm_y, 0, NC * d * sizeof(bf16)));
+        bool ok = make_tmap_bf16_2d(&m->t_lm, m->lm_head, c.vocab, d, d, kGemmBN) == 0;
+        ok = ok && make_tmap_bf16_2d(&m->t_lm_h, m->lm_head, c.vocab, d, d, 128) == 0;
+        ok = ok && make_tmap_bf16_2d(&m->t_tm_y, m->tm_y, NC, d, d, kGemmBM) == 0;
+        if (!ok) return VERILLM_E_CUDA;
+    }
+    if ((rc = copy_in(m->lm_head, lm_head, static_cast<size_t>(c.vocab) * d * sizeof(bf16), on_device))) return rc;
+    CU_TRY(cudaDeviceSynchronize());
+    return VERILLM_OK;
+}
+
+int verillm_token_match(verillm_model* m, const float* last_hidden, const int32_t* claimed, int32_t n_check,
+                        int32_t* argmax_out, uint8_t* match_out, float* margin_out, void* cuda_stream) {
+    if (!m || !last_hidden || !claimed || !argmax_out || !match_out || !margin_out || n_check < 1) return VERILLM_E_INVAL;
+    if (!m->lm_head) return VERILLM_E_INVAL;  // verillm_load_lm_head first
+    if (n_check > m->cfg.max_checks) return VERILLM_E_SHAPE;
+    const verillm_config& c = m->cfg;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    CU_TRY(cudaMemcpyAsync(m->tm_claimed, claimed, sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+    CU_TRY(launch_rmsnorm(last_hidden, m->final_norm, m->tm_y, n_check, c.d_model, c.rms_eps, st));
+    GemmParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = n_check; p.N = c.vocab; p.K = c.d_model; p.out = m->tm_rec; p.ldo = 0; p.status = m->status;
+    p.pair = use_pair(n_check);
+    CU_TRY(cudaMemsetAsync(m->status, 0, sizeof(int), st));
+    CU_TRY(launch_gemm(EPI_ARGMAX, m->t_tm_y, p.pair ? m->t_lm_h : m->t_lm, p, m->num_sms, st));
+    CU_TRY(launch_argmax_reduce(m->tm_rec, n_check, m->n_tiles_v, m->tm_claimed, argmax_out, match_out, margin_out, st));
     return VERILLM_OK;
 }
 

@@ -276,6 +276,14 @@ def final_norm_weights(
     return normal_tensor(wl.seed, 2, (wl.shape.d_model,), _GAMMA_STD, 1.0, device, dtype)
 
 
+def lm_head_weights(
+    wl: Workload, device: torch.device | str = "cpu", dtype: torch.dtype = torch.bfloat16
+) -> torch.Tensor:
+    """Output head [vocab, d_model] (untied from the embedding)."""
+    s = wl.shape
+    return normal_tensor(wl.seed, 3, (s.vocab, s.d_model), weight_std(s), 0.0, device, dtype)
+
+
 def model_weights(
     wl: Workload, device: torch.device | str = "cpu", dtype: torch.dtype = torch.bfloat16
 ) -> Dict[str, object]:

@@ -250,3 +250,42 @@ def test_llama8b_width_reduced_depth():
     assert g["pos_ok"].tolist() == [1, 1, 1, 0, 1, 1] and g["seq_ok"].tolist() == [1, 1, 0]
     assert g["first_bad_layer"][3] == 1
     model.close()
+
+
+def test_tail_token_match_same_states_and_end_to_end(small):
+    """Arg-max of the output head on the last-layer states against the oracle: on identical states (single-CTA
+    and CTA-pair product), and end to end on the states each side recomputed itself."""
+    wl, tokens, om, cs, cp, committed, model, rng, _ = small
+    lm = synth.lm_head_weights(wl, DEV)
+    model.load_lm_head(lm)
+    lm64 = vo.as_f64(H.bits(lm))
+    wide = H.gpu_model(wl, 256)  # a handle sized for more checked rows than the configured 1 %
+    wide.load_lm_head(lm)
+    # (a) identical inputs: oracle last-layer states of 200 positions (pair kernel) and of 20 (single CTA)
+    states = [vo.forward_prefill(om, tokens[b][:256])[-1] for b in range(2)]
+    last = np.concatenate(states)[::2][:200].astype(np.float32)
+    arg_o, _, margin_o = vo.token_match(om, last.astype(np.float64), lm64, np.zeros(len(last), np.int64))
+    claimed = arg_o.copy()
+    forged = [3, 77, 150]
+    claimed[forged] = (claimed[forged] + 1) % wl.shape.vocab
+    for n in (200, 20):
+        arg, match, margin = wide.token_match(torch.from_numpy(last[:n]).to(DEV), claimed[:n])
+        arg, match, margin = arg.cpu().numpy(), match.cpu().numpy(), margin.cpu().numpy()
+        clear = margin_o[:n] > 5e-3  # bf16 rounding of the normed state moves logits by ~1e-3 here
+        assert clear.mean() > 0.8
+        assert np.array_equal(arg[clear], arg_o[:n][clear])
+        want = (arg_o[:n] == claimed[:n]).astype(np.uint8)
+        assert np.array_equal(match[clear], want[clear])
+        assert all(match[i] == 0 for i in forged if i < n and clear[i])
+        assert np.all(np.abs(margin - margin_o[:n])[clear] <= 5e-3)
+    wide.close()
+    # (b) end to end: each side uses the last-layer states it recomputed at the checked positions
+    g, o = run_both(model, om, wl, tokens, committed, cs, cp, prefix_only=True)
+    arg_o, _, margin_o = vo.token_match(om, o.hidden[-1], lm64, np.zeros(len(cs), np.int64))
+    h_last = torch.from_numpy(np.ascontiguousarray(g["hidden"][-1])).to(DEV)
+    arg, match, _ = model.token_match(h_last, arg_o)
+    clear = margin_o > 3e-2  # states differ by up to 2e-2 relative
+    assert clear.sum() >= len(cs) // 2
+    assert np.array_equal(arg.cpu().numpy()[clear], arg_o[clear]) and match.cpu().numpy()[clear].all()
+    with pytest.raises(vb.VerillmError):
+        model.token_match(torch.zeros(len(cs) + 1, wl.shape.d_model, device=DEV), np.zeros(len(cs) + 1, np.int32))

@@ -371,3 +371,43 @@ def test_synth_generator_is_reproducible_and_distributed_as_stated():
     rows = synth.embed_weights(wl, rows=torch.tensor([5, 1000]))
     full = synth.embed_weights(wl)
     assert torch.equal(rows, full[[5, 1000]])
+
+
+def test_token_match_against_transformers_causal_lm():
+    """Final norm + output head + arg-max against the library's causal-LM logits."""
+    from transformers import LlamaConfig, LlamaForCausalLM
+
+    shape = synth.ModelShape(2, 64, 4, 2, 16, 96, 211, 10000.0, 1e-5)
+    m = random_model(shape, 21, std=0.15)
+    rng = np.random.default_rng(22)
+    lm_head = 0.2 * rng.standard_normal((shape.vocab, shape.d_model))
+    cfg = LlamaConfig(
+        vocab_size=shape.vocab, hidden_size=shape.d_model, intermediate_size=shape.d_ffn,
+        num_hidden_layers=shape.n_layers, num_attention_heads=shape.n_heads, num_key_value_heads=shape.n_kv_heads,
+        head_dim=shape.head_dim, rms_norm_eps=shape.rms_eps, rope_theta=shape.rope_base, attention_bias=False,
+        mlp_bias=False, max_position_embeddings=256, tie_word_embeddings=False,
+    )
+    hf = LlamaForCausalLM(cfg).double().eval()
+    names = {"attn_norm": "input_layernorm", "wq": "self_attn.q_proj", "wk": "self_attn.k_proj",
+             "wv": "self_attn.v_proj", "wo": "self_attn.o_proj", "ffn_norm": "post_attention_layernorm",
+             "w_gate": "mlp.gate_proj", "w_up": "mlp.up_proj", "w_down": "mlp.down_proj"}
+    sd = {"model.embed_tokens.weight": m.embed, "model.norm.weight": m.final_norm, "lm_head.weight": lm_head}
+    for l, lw in enumerate(m.layers):
+        for k, v in lw.items():
+            sd[f"model.layers.{l}.{names[k]}.weight"] = v
+    missing = hf.load_state_dict({k: torch.from_numpy(np.ascontiguousarray(v)) for k, v in sd.items()}, strict=False)
+    assert not [k for k in missing.missing_keys if "rotary" not in k]
+    toks = rng.integers(0, shape.vocab, 29)
+    with torch.no_grad():
+        ref_logits = hf(input_ids=torch.from_numpy(toks)[None], use_cache=False).logits[0].numpy()
+    last = vo.forward_prefill(m, toks)[-1]
+    claimed = np.argmax(ref_logits, axis=-1)
+    claimed[5] = (claimed[5] + 1) % shape.vocab  # one forged token
+    arg, match, margin = vo.token_match(m, last, lm_head, claimed)
+    assert np.array_equal(arg, np.argmax(ref_logits, axis=-1))
+    assert match.tolist() == [0 if i == 5 else 1 for i in range(29)]
+    srt = np.sort(ref_logits, axis=-1)
+    assert np.allclose(margin, srt[:, -1] - srt[:, -2], rtol=0, atol=2e-5)  # the library keeps its rotary table in float32
+    # a duplicated head row ties (up to the summation order of the matrix product): margin vanishes
+    a2, _, m2 = vo.token_match(m, last[:1], np.concatenate([lm_head[:3], lm_head[:3]]), np.array([0]))
+    assert a2[0] % 3 == int(np.argmax(lm_head[:3] @ vo.rmsnorm(last[0], m.final_norm, m.rms_eps))) and m2[0] < 1e-12
