@@ -198,21 +198,31 @@ def layer_forward(m: Model, w: Dict[str, np.ndarray], h: np.ndarray, positions: 
     return u + (silu(f @ w["w_gate"].T) * (f @ w["w_up"].T)) @ w["w_down"].T
 
 
+def forward_segment_batch(m: Model, states_in: Sequence[np.ndarray], layer_begin: int, layer_end: int) -> List[np.ndarray]:
+    """Segment-local pass: S_{i+1}^{(t)} = F_i(S_i^{(t)}; W_i) for all t, for the blocks layer_begin .. layer_end-1,
+    starting from given input states (one [T_b, d_model] array per sequence: the recorded upstream states
+    of a verifier's segment, or the embeddings for the first segment).
+
+    Returns one [layer_end - layer_begin, T_b, d_model] array per sequence.  Sequences never interact; the
+    loop runs layer by layer over all of them only so that `m.layers` may be a lazy sequence that
+    materialises one layer's weights at a time."""
+    hs = [np.array(h, dtype=np.float64, copy=True) for h in states_in]
+    n = layer_end - layer_begin
+    out = [np.empty((n, h.shape[0], m.d_model), dtype=np.float64) for h in hs]
+    for l in range(layer_begin, layer_end):
+        w = m.layers[l]
+        for b in range(len(hs)):
+            hs[b] = layer_forward(m, w, hs[b], np.arange(hs[b].shape[0]))
+            out[b][l - layer_begin] = hs[b]
+    return out
+
+
 def forward_prefill_batch(m: Model, seqs: Sequence[np.ndarray]) -> List[np.ndarray]:
     """All layer-output states of every sequence, each in a single causal pass (Eq. 1).
 
     Returns one [n_layers, T_b, d_model] array per sequence: entry l is the residual stream after
-    block l+1, i.e. the boundary state S_{l+2} in the paper's numbering, before the final norm.
-    Sequences never interact; the loop runs layer by layer over all of them only so that `m.layers`
-    may be a lazy sequence that materialises one layer's weights at a time."""
-    hs = [embed_tokens(m, np.asarray(t)) for t in seqs]
-    out = [np.empty((m.n_layers, len(t), m.d_model), dtype=np.float64) for t in seqs]
-    for l in range(m.n_layers):
-        w = m.layers[l]
-        for b in range(len(seqs)):
-            hs[b] = layer_forward(m, w, hs[b], np.arange(hs[b].shape[0]))
-            out[b][l] = hs[b]
-    return out
+    block l+1, i.e. the boundary state S_{l+2} in the paper's numbering, before the final norm."""
+    return forward_segment_batch(m, [embed_tokens(m, np.asarray(t)) for t in seqs], 0, m.n_layers)
 
 
 def forward_prefill(m: Model, tokens: np.ndarray) -> np.ndarray:
@@ -402,6 +412,25 @@ def verdict(stats: np.ndarray, check_seq: np.ndarray, batch: int, tol: Tol):
             seq_ok[b] = np.uint8(np.all(pos_ok[sel]))
             seq_score[b] = float(np.mean(stats[sel][:, :, mae_idx]))
     return pos_ok.astype(np.uint8), first_bad, seq_ok, seq_score
+
+
+def verify_segment(
+    m: Model, states_in: Sequence[np.ndarray], layer_begin: int, layer_end: int, committed: np.ndarray,
+    check_seq: np.ndarray, check_pos: np.ndarray, tol: Tol, commit_dtype: str = "bf16",
+) -> Report:
+    """Segment verifier: recompute blocks layer_begin .. layer_end-1 from the recorded upstream states of every
+    position, compare at the checked positions with the committed outputs [layer_end - layer_begin, n_check,
+    d_model] and decide.  Layer indices in the report count from layer_begin."""
+    committed = as_f64(committed)
+    n_check = len(check_seq)
+    n = layer_end - layer_begin
+    hidden = np.zeros((n, n_check, m.d_model), dtype=np.float64)
+    outs = forward_segment_batch(m, states_in, layer_begin, layer_end)
+    for slot in range(n_check):
+        hidden[:, slot, :] = outs[int(check_seq[slot])][:, int(check_pos[slot]), :]
+    stats = np.transpose(compare_stats(hidden, committed, commit_dtype, tol), (1, 0, 2)).copy()
+    pos_ok, first_bad, seq_ok, seq_score = verdict(stats, np.asarray(check_seq), len(states_in), tol)
+    return Report(stats, pos_ok, first_bad, seq_ok, seq_score, hidden)
 
 
 def token_match(m: Model, last_hidden: np.ndarray, lm_head: np.ndarray, claimed: np.ndarray):

@@ -411,3 +411,29 @@ def test_token_match_against_transformers_causal_lm():
     # a duplicated head row ties (up to the summation order of the matrix product): margin vanishes
     a2, _, m2 = vo.token_match(m, last[:1], np.concatenate([lm_head[:3], lm_head[:3]]), np.array([0]))
     assert a2[0] % 3 == int(np.argmax(lm_head[:3] @ vo.rmsnorm(last[0], m.final_norm, m.rms_eps))) and m2[0] < 1e-12
+
+
+def test_segments_compose_to_the_full_pass():
+    """Running blocks [0, a) and then [a, L) from the first segment's output reproduces the single pass bit
+    for bit, and a segment's result depends only on its input states."""
+    shape = small_shape(n_layers=4)
+    m = random_model(shape, 23)
+    rng = np.random.default_rng(24)
+    seqs = [rng.integers(0, shape.vocab, 11), rng.integers(0, shape.vocab, 6)]
+    full = vo.forward_prefill_batch(m, seqs)
+    first = vo.forward_segment_batch(m, [vo.embed_tokens(m, t) for t in seqs], 0, 3)
+    second = vo.forward_segment_batch(m, [f[-1] for f in first], 3, 4)
+    for b in range(2):
+        assert np.array_equal(np.concatenate([first[b], second[b]]), full[b])
+    # verify_segment on its own outputs accepts with zero deviation; a perturbed upstream state is caught downstream
+    cs, cp = np.array([0, 1, 0]), np.array([10, 2, 4])
+    own = np.stack([second[s][:, p] for s, p in zip(cs, cp)], axis=1)
+    rep = vo.verify_segment(m, [f[-1] for f in first], 3, 4, own, cs, cp, vo.Tol(), "f32")
+    assert rep.pos_ok.all() and rep.stats[..., 0].max() < 1e-6
+    bad_in = [f[-1].copy() for f in first]
+    bad_in[0][4] *= 1.5
+    rep = vo.verify_segment(m, bad_in, 3, 4, own, cs, cp, vo.Tol(), "f32")
+    rel = rep.stats[:, 0, 0]
+    assert rep.pos_ok[2] == 0 and rel[2] > 0.1  # the perturbed position itself
+    assert rel[1] < 1e-6  # another sequence: untouched
+    assert 1e-6 < rel[0] < rel[2]  # a later position of the same sequence attends to it and moves, but less
