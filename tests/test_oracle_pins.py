@@ -431,7 +431,7 @@ def test_segments_compose_to_the_full_pass():
     rep = vo.verify_segment(m, [f[-1] for f in first], 3, 4, own, cs, cp, vo.Tol(), "f32")
     assert rep.pos_ok.all() and rep.stats[..., 0].max() < 1e-6
     bad_in = [f[-1].copy() for f in first]
-    bad_in[0][4] *= 1.5
+    bad_in[0][4] += rng.standard_normal(shape.d_model) * np.sqrt(np.mean(bad_in[0][4] ** 2))  # not a rescaling: the norm would undo it
     rep = vo.verify_segment(m, bad_in, 3, 4, own, cs, cp, vo.Tol(), "f32")
     rel = rep.stats[:, 0, 0]
     assert rep.pos_ok[2] == 0 and rel[2] > 0.1  # the perturbed position itself
