@@ -160,6 +160,20 @@ int verillm_verify_prefill(verillm_model *model, const int32_t *tokens, const in
                            const int32_t *check_pos, int32_t n_check, const verillm_tol *tol,
                            const verillm_report *report, void *cuda_stream);
 
+/* Segment-local verification ("for segment i, the verifier uses the recorded upstream hidden states as its inputs
+ * and executes only its own block of layers"; T_verify ~ T_prefill / L): blocks layer_begin .. layer_end-1 are
+ * recomputed for all positions from the recorded states entering block layer_begin, and compared at the checked
+ * positions with the committed outputs of those blocks.
+ *  input_states     DEVICE [cu_seqlens[batch]][d_model] in input_dtype (BF16 / F32): the residual stream entering
+ *                   block layer_begin at every position (the output of block layer_begin-1, or the embeddings)
+ *  committed_hidden DEVICE [layer_end - layer_begin][n_check][d_model]
+ * The report arrays have layer_end - layer_begin layers and their layer indices count from layer_begin; all else
+ * as verillm_verify_prefill.  Extra errors: E_RANGE for an empty or out-of-range layer interval. */
+int verillm_verify_segment(verillm_model *model, const void *input_states, int32_t input_dtype, int32_t layer_begin,
+                           int32_t layer_end, const int32_t *cu_seqlens, int32_t batch, const void *committed_hidden,
+                           int32_t commit_dtype, const int32_t *check_seq, const int32_t *check_pos, int32_t n_check,
+                           const verillm_tol *tol, const verillm_report *report, void *cuda_stream);
+
 /* The prover's side, for generating traces: teacher-forced token-by-token decode with a bf16
  * key/value cache (the decode loop of the Inference Scheme), after an optional parallel pass over the
  * first n_prefill tokens of every sequence.  Writes the layer-output states at the requested

@@ -30,7 +30,7 @@ EXPORTS = (
     "verillm_verify_prefill", "verillm_decode_commit", "verillm_compare", "verillm_compare_noalloc", "verillm_op_gemm",
     "verillm_op_rmsnorm", "verillm_op_attention", "verillm_free", "verillm_strerror",
     "verillm_last_launch_count", "verillm_profile_enable", "verillm_profile_read",
-    "verillm_load_lm_head", "verillm_token_match",
+    "verillm_load_lm_head", "verillm_token_match", "verillm_verify_segment",
 )
 PROF_CLASSES = ("setup", "rmsnorm", "gemm_qkv_rope", "attention", "gemm_o_resid", "gemm_gate_up_swiglu",
                 "gemm_down_resid_compare", "verdict")
@@ -109,6 +109,11 @@ def lib() -> C.CDLL:
         ]
         L.verillm_compare_noalloc.argtypes = L.verillm_compare.argtypes
         L.verillm_compare_noalloc.restype = C.c_int
+        L.verillm_verify_segment.argtypes = [
+            C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32,
+            C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(Tol), C.POINTER(ReportC), C.c_void_p,
+        ]
+        L.verillm_verify_segment.restype = C.c_int
         L.verillm_load_lm_head.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
         L.verillm_load_lm_head.restype = C.c_int
         L.verillm_token_match.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -260,6 +265,28 @@ class Model:
                 self._h, tokens.data_ptr(), cu.ctypes.data, batch, _ptr(committed), dtype, cs.ctypes.data, cp.ctypes.data,
                 n_check, C.byref(tol), C.byref(rc_struct), _stream_ptr(stream))
         _check(code, "verillm_verify_prefill")
+        return report
+
+    def verify_segment(self, input_states: torch.Tensor, layer_begin: int, layer_end: int, cu_seqlens: Sequence[int],
+                       committed: Optional[torch.Tensor], check_seq: Sequence[int], check_pos: Sequence[int],
+                       tol: Optional[Tol] = None, want_hidden: bool = False,
+                       stream: Optional[torch.cuda.Stream] = None) -> Report:
+        """input_states: device [n_tokens][d_model] bf16/f32; committed: device [layer_end-layer_begin][n_check][d_model]."""
+        cu = _i32(cu_seqlens)
+        cs, cp = _i32(check_seq), _i32(check_pos)
+        n_check, batch = int(cs.shape[0]), int(cu.shape[0]) - 1
+        tol = tol or default_tol()
+        report = Report(n_check, layer_end - layer_begin, batch, self.shape.d_model, self.device, want_hidden)
+        if not input_states.is_contiguous() or input_states.dtype not in (torch.bfloat16, torch.float32):
+            raise ValueError("input states must be contiguous bf16 or float32")
+        cdt = BF16 if committed is None or committed.dtype == torch.bfloat16 else F32
+        st = report.c_struct()
+        with torch.cuda.device(self.device):
+            code = lib().verillm_verify_segment(
+                self._h, input_states.data_ptr(), BF16 if input_states.dtype == torch.bfloat16 else F32, layer_begin,
+                layer_end, cu.ctypes.data, batch, _ptr(committed), cdt, cs.ctypes.data, cp.ctypes.data, n_check,
+                C.byref(tol), C.byref(st), _stream_ptr(stream))
+        _check(code, "verillm_verify_segment")
         return report
 
     def decode_commit(self, tokens: torch.Tensor, cu_seqlens: Sequence[int], n_prefill: int, check_seq: Sequence[int],

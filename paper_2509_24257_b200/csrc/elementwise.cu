@@ -444,6 +444,19 @@ __global__ void convert_states_kernel(const float* __restrict__ src, void* __res
     else reinterpret_cast<float*>(dst)[i] = src[i];
 }
 
+__global__ void load_states_kernel(const void* __restrict__ src, int dtype, size_t n, float* __restrict__ dst) {
+    const size_t i = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
+    if (i >= n) return;  // n is a multiple of 4 (d_model % 64 == 0)
+    float4 v;
+    if (dtype == VERILLM_BF16) {
+        const uint2 u = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(src) + i);
+        v = make_float4(bf16_lo(u.x), bf16_hi(u.x), bf16_lo(u.y), bf16_hi(u.y));
+    } else {
+        v = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(src) + i);
+    }
+    *reinterpret_cast<float4*>(dst + i) = v;
+}
+
 __global__ void gather_tokens_kernel(const int* __restrict__ tokens, const int* __restrict__ src_index, int n,
                                      int* __restrict__ out) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -579,6 +592,12 @@ cudaError_t launch_scatter_kv(const void* qkv, const int* dst_row, int rows, int
 cudaError_t launch_convert_states(const float* src, void* dst, size_t n, int commit_dtype, cudaStream_t s) {
     if (n == 0) return cudaSuccess;
     convert_states_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, s>>>(src, dst, n, commit_dtype);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_load_states(const void* src, int dtype, size_t n, float* resid, cudaStream_t s) {
+    if (n == 0) return cudaSuccess;
+    load_states_kernel<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, s>>>(src, dtype, n, resid);
     return cudaGetLastError();
 }
 

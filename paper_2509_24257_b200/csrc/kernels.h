@@ -68,6 +68,8 @@ cudaError_t launch_slot_lists(const int* tok_of_slot, int n_check, int n_tokens,
                               cudaStream_t stream);
 cudaError_t launch_embed(const int* tokens, const void* table, int n_tokens, int d_model, int vocab, float* resid,
                          int* status, cudaStream_t stream);
+// resid[n] (fp32) = recorded states in `dtype` (VERILLM_BF16 / VERILLM_F32): input of a segment-local pass
+cudaError_t launch_load_states(const void* src, int dtype, size_t n, float* resid, cudaStream_t stream);
 cudaError_t launch_rmsnorm(const float* x, const void* gain, void* y, int rows, int d, float eps,
                            cudaStream_t stream);
 cudaError_t launch_compare_rows(const float* hidden, const void* committed, int n_rows, int d, const CmpParams& cmp,

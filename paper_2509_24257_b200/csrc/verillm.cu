@@ -496,11 +496,14 @@ int verillm_load_weights(const verillm_config* cfg, const verillm_weights* weigh
     return VERILLM_OK;
 }
 
-int verillm_verify_prefill(verillm_model* m, const int32_t* tokens, const int32_t* cu_seqlens, int32_t batch,
-                           const void* committed_hidden, int32_t commit_dtype, const int32_t* check_seq,
-                           const int32_t* check_pos, int32_t n_check, const verillm_tol* tol,
-                           const verillm_report* rep, void* cuda_stream) {
-    if (!m || !tokens || !tol || !rep) return VERILLM_E_INVAL;
+// Shared body of the full verifier (tokens in, blocks 0 .. n_layers-1) and the segment verifier (recorded
+// upstream states in, blocks l0 .. l1-1).  Exactly one of tokens / states_in is given.
+static int verify_impl(verillm_model* m, const int32_t* tokens, const void* states_in, int32_t in_dtype, int l0, int l1,
+                       const int32_t* cu_seqlens, int32_t batch, const void* committed_hidden, int32_t commit_dtype,
+                       const int32_t* check_seq, const int32_t* check_pos, int32_t n_check, const verillm_tol* tol,
+                       const verillm_report* rep, void* cuda_stream) {
+    if (!m || (!tokens && !states_in) || !tol || !rep) return VERILLM_E_INVAL;
+    if (l0 < 0 || l1 > m->cfg.n_layers || l0 >= l1) return VERILLM_E_RANGE;
     if (commit_dtype != VERILLM_BF16 && commit_dtype != VERILLM_F32) return VERILLM_E_INVAL;
     if (!rep->seq_ok || !rep->seq_score || !rep->status) return VERILLM_E_INVAL;
     if (n_check > 0 && (!committed_hidden || !rep->stats || !rep->pos_ok || !rep->first_bad_layer)) return VERILLM_E_INVAL;
@@ -522,7 +525,10 @@ int verillm_verify_prefill(verillm_model* m, const int32_t* tokens, const int32_
     }
     CU_TRY(launch_token_maps(m->cu_dev, batch, M, m->pos_of_token, m->seq_of_token, st));
     CU_TRY(launch_slot_lists(m->tok_of_slot, n_check, M, m->slot_first, m->slot_next, st));
-    CU_TRY(launch_embed(tokens, m->embed, M, c.d_model, c.vocab, m->resid, rep->status, st));
+    if (tokens)
+        CU_TRY(launch_embed(tokens, m->embed, M, c.d_model, c.vocab, m->resid, rep->status, st));
+    else
+        CU_TRY(launch_load_states(states_in, in_dtype, static_cast<size_t>(M) * c.d_model, m->resid, st));
     launches += 2 + (n_check > 0 ? 1 : 0);
     prof_mark(m, VERILLM_PROF_SETUP, st);
 
@@ -532,21 +538,40 @@ int verillm_verify_prefill(verillm_model* m, const int32_t* tokens, const int32_
     cl.slot_first = m->slot_first; cl.slot_next = m->slot_next; cl.n_check = n_check;
     cl.cmp = cmp_params(*tol, commit_dtype);
     LayerRun run{M, batch, max_len, m->cu_dev, n_check > 0 ? &cl : nullptr};
-    for (int l = 0; l < c.n_layers; ++l) {
-        const size_t slab = static_cast<size_t>(l) * n_check;
+    for (int l = l0; l < l1; ++l) {
+        const size_t slab = static_cast<size_t>(l - l0) * n_check;
         cl.committed = reinterpret_cast<const char*>(committed_hidden) + slab * c.d_model * e_commit;
         cl.partials = m->partials + slab * m->n_tiles_d * kNPart;
         cl.hidden_out = rep->hidden_out ? rep->hidden_out + slab * c.d_model : nullptr;
         if ((rc = run_layer(m, l, run, rep->status, st, &launches))) return rc;
     }
-    CU_TRY(launch_verdict(m->partials, c.n_layers, n_check, m->n_tiles_d, c.d_model, tol_dev(*tol), rep->status,
+    CU_TRY(launch_verdict(m->partials, l1 - l0, n_check, m->n_tiles_d, c.d_model, tol_dev(*tol), rep->status,
                           rep->stats, rep->pos_ok, rep->first_bad_layer, st));
-    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, m->seq_of_slot, n_check, c.n_layers, batch, rep->seq_ok,
+    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, m->seq_of_slot, n_check, l1 - l0, batch, rep->seq_ok,
                               rep->seq_score, st));
     launches += (n_check > 0 ? 1 : 0) + 1;
     prof_mark(m, VERILLM_PROF_VERDICT, st);
     m->last_launches = launches;
     return VERILLM_OK;
+}
+
+int verillm_verify_prefill(verillm_model* m, const int32_t* tokens, const int32_t* cu_seqlens, int32_t batch,
+                           const void* committed_hidden, int32_t commit_dtype, const int32_t* check_seq,
+                           const int32_t* check_pos, int32_t n_check, const verillm_tol* tol,
+                           const verillm_report* rep, void* cuda_stream) {
+    if (!m || !tokens) return VERILLM_E_INVAL;
+    return verify_impl(m, tokens, nullptr, VERILLM_BF16, 0, m->cfg.n_layers, cu_seqlens, batch, committed_hidden,
+                       commit_dtype, check_seq, check_pos, n_check, tol, rep, cuda_stream);
+}
+
+int verillm_verify_segment(verillm_model* m, const void* input_states, int32_t input_dtype, int32_t layer_begin,
+                           int32_t layer_end, const int32_t* cu_seqlens, int32_t batch, const void* committed_hidden,
+                           int32_t commit_dtype, const int32_t* check_seq, const int32_t* check_pos, int32_t n_check,
+                           const verillm_tol* tol, const verillm_report* rep, void* cuda_stream) {
+    if (!m || !input_states) return VERILLM_E_INVAL;
+    if (input_dtype != VERILLM_BF16 && input_dtype != VERILLM_F32) return VERILLM_E_INVAL;
+    return verify_impl(m, nullptr, input_states, input_dtype, layer_begin, layer_end, cu_seqlens, batch,
+                       committed_hidden, commit_dtype, check_seq, check_pos, n_check, tol, rep, cuda_stream);
 }
 
 int verillm_compare(const float* hidden, const void* committed, int32_t commit_dtype, int32_t n_layers, int32_t n_check,

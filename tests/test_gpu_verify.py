@@ -289,3 +289,26 @@ def test_tail_token_match_same_states_and_end_to_end(small):
     assert np.array_equal(arg.cpu().numpy()[clear], arg_o[clear]) and match.cpu().numpy()[clear].all()
     with pytest.raises(vb.VerillmError):
         model.token_match(torch.zeros(len(cs) + 1, wl.shape.d_model, device=DEV), np.zeros(len(cs) + 1, np.int32))
+
+
+def test_segment_local_verification_matches_oracle(small):
+    """Blocks 2..3 recomputed from the recorded states entering block 2 (all positions), as a segment verifier
+    does; committed outputs from the oracle's own segment pass, one of them tampered."""
+    wl, tokens, om, cs, cp, _, model, rng, _ = small
+    full = vo.forward_prefill_batch(om, list(tokens))
+    upstream = [vo.round_to_bf16(f[1]) for f in full]  # recorded S entering block 2, serialised as bf16
+    outs = vo.forward_segment_batch(om, upstream, 2, 4)
+    honest = np.stack([outs[s][:, p] for s, p in zip(cs, cp)], axis=1)
+    tampered = synth.add_state_noise(honest, [4], [1], 10 * TOL, rng)
+    comm_t = synth.to_commit_dtype(tampered, "bf16")
+    states = synth.to_commit_dtype(np.concatenate(upstream), "bf16").to(DEV)
+    rep = model.verify_segment(states, 2, 4, synth.cu_seqlens(wl), comm_t.to(DEV), cs, cp, want_hidden=True)
+    g = rep.cpu()
+    o = vo.verify_segment(om, upstream, 2, 4, comm_t.to(torch.float64).numpy(), cs, cp, vo.Tol(), "bf16")
+    assert g["stats"].shape == (len(cs), 2, vb.NSTAT)
+    assert_parity(g, o, expect_reject=[4])
+    assert g["first_bad_layer"][4] == 1 and g["pos_ok"].sum() == len(cs) - 1  # index counted from layer_begin
+    # the same entry point from the embeddings reproduces the full pass over the first blocks
+    with pytest.raises(vb.VerillmError) as e:
+        model.verify_segment(states, 3, 3, synth.cu_seqlens(wl), comm_t.to(DEV), cs, cp)
+    assert e.value.code == vb.E_RANGE
