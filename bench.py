@@ -353,6 +353,27 @@ def run_ours(args, wl):
                    "achieved_gbs": round(tm_bytes / (tm_ms * 1e-3) / 1e9, 1), "peak_gbs": peaks["hbm_gbs"],
                    "frac": round(tm_bytes / (tm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
 
+    # ---- the comparison path alone at full coverage (every position of 2 sequences checked at every layer):
+    # the standalone compare + verdict kernels stream hidden (fp32) and committed (bf16) states once
+    n_rows = min(2 * wl.seq_len, wl.n_tokens)
+    hid = torch.randn(s.n_layers, n_rows, s.d_model, device=device)
+    com = (hid * (1 + 4e-3 * torch.randn_like(hid))).to(torch.bfloat16)
+    seq_of = (np.arange(n_rows) // wl.seq_len).astype(np.int32)
+    for _ in range(2):
+        vb.compare(hid, com, seq_of, 2, tol, stream)
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    c0.record(stream)
+    for _ in range(5):
+        vb.compare(hid, com, seq_of, 2, tol, stream)
+    c1.record(stream)
+    torch.cuda.synchronize()
+    cmp_ms = c0.elapsed_time(c1) / 5
+    cmp_bytes = hid.numel() * 6
+    compare_path = {"rows": int(s.n_layers * n_rows), "ms": round(cmp_ms, 4), "bound": "hbm",
+                    "achieved_gbs": round(cmp_bytes / (cmp_ms * 1e-3) / 1e9, 1), "peak_gbs": peaks["hbm_gbs"],
+                    "frac": round(cmp_bytes / (cmp_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
+    del hid, com
+
     if rank == 0:
         run, desc = oracle_sample(wl, 12.0, str(device)) if args.gpus == 1 else (None, None)
         cpu_baseline = None
@@ -379,7 +400,7 @@ def run_ours(args, wl):
                          "status": res["status"]},
             "clocks": clocks, "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                                      "d2h_bytes_per_step": int(d2h)},
-            "gpu_launches": int(launches), "roofline": roofline, "token_match": token_match,
+            "gpu_launches": int(launches), "roofline": roofline, "token_match": token_match, "compare_path": compare_path,
             "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))

@@ -2,8 +2,8 @@
 // softmax(q k^T / sqrt(dh) + causal mask) v, flash style ("a single forward pass under the causal mask").
 //
 // One CTA owns 128 query rows of one (sequence, query head) and walks the key/value tiles of 64 positions
-// up to the diagonal.  Warp 4 (one thread) drives everything asynchronous: TMA loads of Q and of a
-// double-buffered K/V ring (128-byte swizzle), S = Q K^T and O += P V as tcgen05.mma into tensor memory.
+// up to the diagonal.  Warp 4 (one thread) drives everything asynchronous: TMA loads of Q and of separate
+// key (3 tiles) and value (2 tiles) rings (128-byte swizzle), S = Q K^T and O += P V as tcgen05.mma.
 // Warps 0-3 own one query row per thread: they read S from TMEM, keep the online softmax (reference
 // maximum and running sum, fp32, exp2) in registers and write P as packed bf16 back over the S columns,
 // from where the second product takes it as its A operand.  O accumulates in TMEM across tiles; it is
@@ -21,6 +21,7 @@ namespace {
 constexpr int TC_BM = 128;
 constexpr int TC_BN = 64;
 constexpr int TC_THREADS = 160;
+constexpr int TC_KSTAGES = 3;  // key tiles in flight (a key tile is free as soon as its Q K^T is done); value tiles: 2
 constexpr int TC_TMEM_COLS = 256;  // S0/P0 [0,64), S1/P1 [64,128), O [128, 128 + dh)
 constexpr float TC_RESCALE_LOG2 = 8.f;  // rescale O when a row maximum exceeds its reference by this (log2)
 
@@ -29,9 +30,9 @@ struct TcSmem {
     static constexpr uint32_t Q_BYTES = TC_BM * DH * 2;
     static constexpr uint32_t KV_BYTES = TC_BN * DH * 2;
     static constexpr uint32_t K_OFF = Q_BYTES;
-    static constexpr uint32_t V_OFF = K_OFF + 2 * KV_BYTES;
+    static constexpr uint32_t V_OFF = K_OFF + TC_KSTAGES * KV_BYTES;
     static constexpr uint32_t BAR_OFF = V_OFF + 2 * KV_BYTES;
-    static constexpr uint32_t TOTAL = BAR_OFF + 128;
+    static constexpr uint32_t TOTAL = BAR_OFF + 256;
 };
 
 // K-major operand whose rows are 128 bytes (64 bf16) with the 128-byte swizzle: see umma_desc_k_sw128.
@@ -52,16 +53,20 @@ __device__ __forceinline__ float ex2(float x) {
 template <int DH>
 __global__ void __launch_bounds__(TC_THREADS, 2)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
-               const int* __restrict__ cu_seqlens, int n_heads, int n_kv_heads, __nv_bfloat16* __restrict__ out,
-               int* status) {
+               const int* __restrict__ cu_seqlens, int batch, int n_qblocks, int n_heads, int n_kv_heads,
+               __nv_bfloat16* __restrict__ out, int* status) {
     using L = TcSmem<DH>;
     constexpr int QB = DH / 64;  // 64-column blocks per head
     extern __shared__ __align__(1024) uint8_t tc_smem[];
 
-    const int seq = blockIdx.z, head = blockIdx.y;
+    // Work order: all (sequence, head) pairs of the last query tile first, then the tile before it, ...: the
+    // CTAs with the most key tiles start first (longest-processing-time order), heads of a KV group adjacent.
+    const int pairs = n_heads * batch;
+    const int qb = n_qblocks - 1 - static_cast<int>(blockIdx.x) / pairs;
+    const int rem = static_cast<int>(blockIdx.x) % pairs;
+    const int seq = rem / n_heads, head = rem % n_heads;
     const int seq_start = cu_seqlens[seq];
     const int len = cu_seqlens[seq + 1] - seq_start;
-    const int qb = static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x);  // longest rows first
     const int q0 = qb * TC_BM;
     if (q0 >= len) return;
     const uint32_t sbase = smem_u32(tc_smem);
@@ -80,12 +85,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const uint32_t bar = sbase + L::BAR_OFF;
     const uint32_t q_full = bar, o_done = bar + 8;
     auto p_ready = [&](int b) { return bar + 16 + 8 * b; };
-    auto kv_full = [&](int b) { return bar + 32 + 8 * b; };
-    auto kv_empty = [&](int b) { return bar + 48 + 8 * b; };
-    auto s_full = [&](int b) { return bar + 64 + 8 * b; };
-    const uint32_t tmem_slot = bar + 80;
-    volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(tc_smem + L::BAR_OFF + 80);
-    volatile int* failed = reinterpret_cast<volatile int*>(tc_smem + L::BAR_OFF + 84);
+    auto s_full = [&](int b) { return bar + 32 + 8 * b; };
+    auto k_full = [&](int b) { return bar + 48 + 8 * b; };
+    auto k_empty = [&](int b) { return bar + 72 + 8 * b; };
+    auto v_full = [&](int b) { return bar + 96 + 8 * b; };
+    auto v_empty = [&](int b) { return bar + 112 + 8 * b; };
+    const uint32_t tmem_slot = bar + 128;
+    volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(tc_smem + L::BAR_OFF + 128);
+    volatile int* failed = reinterpret_cast<volatile int*>(tc_smem + L::BAR_OFF + 132);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -94,9 +101,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         mbar_init(o_done, 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(p_ready(b), 128);
-            mbar_init(kv_full(b), 1);
-            mbar_init(kv_empty(b), 1);
             mbar_init(s_full(b), 1);
+            mbar_init(v_full(b), 1);
+            mbar_init(v_empty(b), 1);
+        }
+        for (int b = 0; b < TC_KSTAGES; ++b) {
+            mbar_init(k_full(b), 1);
+            mbar_init(k_empty(b), 1);
         }
         fence_mbar_init();
     }
@@ -113,43 +124,54 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         // ------------------------------------------------------------ TMA + MMA driver (one thread)
         if (lane == 0) {
             bool ok = true;
-            auto load_kv = [&](int j) {
-                const int b = j & 1;
-                mbar_arrive_expect_tx(kv_full(b), 2 * L::KV_BYTES);
+            auto load_k = [&](int j) {
+                const int kb = j % TC_KSTAGES;
+                mbar_arrive_expect_tx(k_full(kb), L::KV_BYTES);
 #pragma unroll
-                for (int c = 0; c < QB; ++c) {
-                    tma_load_2d(k_s(b) + c * (TC_BN * 128), &tmap_kv, dq + kvh * DH + c * 64, seq_start + j * TC_BN, kv_full(b));
-                    tma_load_2d(v_s(b) + c * (TC_BN * 128), &tmap_kv, dq + dkv + kvh * DH + c * 64, seq_start + j * TC_BN, kv_full(b));
-                }
+                for (int c = 0; c < QB; ++c)
+                    tma_load_2d(k_s(kb) + c * (TC_BN * 128), &tmap_kv, dq + kvh * DH + c * 64, seq_start + j * TC_BN, k_full(kb));
+            };
+            auto load_v = [&](int j) {
+                const int b = j & 1;
+                mbar_arrive_expect_tx(v_full(b), L::KV_BYTES);
+#pragma unroll
+                for (int c = 0; c < QB; ++c)
+                    tma_load_2d(v_s(b) + c * (TC_BN * 128), &tmap_kv, dq + dkv + kvh * DH + c * 64, seq_start + j * TC_BN, v_full(b));
             };
             auto issue_qk = [&](int j) {  // S[j & 1] = Q K_j^T : M 128, N 64, K = DH
-                const int b = j & 1;
+                const int b = j & 1, kb = j % TC_KSTAGES;
                 constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, TC_BN);
 #pragma unroll
                 for (int kk = 0; kk < DH / 16; ++kk) {
                     const uint64_t a = umma_desc_k_sw128(q_s + (kk / 4) * (TC_BM * 128)) + 2u * (kk % 4);
-                    const uint64_t bd = umma_desc_k_sw128(k_s(b) + (kk / 4) * (TC_BN * 128)) + 2u * (kk % 4);
+                    const uint64_t bd = umma_desc_k_sw128(k_s(kb) + (kk / 4) * (TC_BN * 128)) + 2u * (kk % 4);
                     umma_bf16(tmem_base + static_cast<uint32_t>(b * TC_BN), a, bd, idesc, kk != 0 ? 1u : 0u);
                 }
                 umma_commit(s_full(b));
+                umma_commit(k_empty(kb));  // the key tile can be replaced once this product is done
             };
             mbar_arrive_expect_tx(q_full, L::Q_BYTES);
 #pragma unroll
             for (int c = 0; c < QB; ++c) tma_load_2d(q_s + c * (TC_BM * 128), &tmap_q, head * DH + c * 64, seq_start + q0, q_full);
-            load_kv(0);
-            if (nb > 1) load_kv(1);
-            ok = mbar_wait(q_full, 0, status) && mbar_wait(kv_full(0), 0, status);
+            for (int j = 0; j < TC_KSTAGES && j < nb; ++j) load_k(j);
+            for (int j = 0; j < 2 && j < nb; ++j) load_v(j);
+            ok = mbar_wait(q_full, 0, status) && mbar_wait(k_full(0), 0, status);
             if (ok) {
                 tc_fence_after();
                 issue_qk(0);
             }
             for (int j = 0; j < nb && ok; ++j) {
                 const int b = j & 1;
-                if (j + 1 < nb) {
-                    if (!mbar_wait(kv_full(b ^ 1), ((j + 1) >> 1) & 1, status)) { ok = false; break; }
+                if (j + 1 < nb) {  // Q K^T runs one tile ahead of the softmax
+                    if (!mbar_wait(k_full((j + 1) % TC_KSTAGES), ((j + 1) / TC_KSTAGES) & 1, status)) { ok = false; break; }
                     tc_fence_after();
                     issue_qk(j + 1);
                 }
+                if (j + TC_KSTAGES < nb) {  // key tile j is consumed (its product was issued an iteration ago): refill
+                    if (!mbar_wait(k_empty(j % TC_KSTAGES), (j / TC_KSTAGES) & 1, status)) { ok = false; break; }
+                    load_k(j + TC_KSTAGES);
+                }
+                if (!mbar_wait(v_full(b), (j >> 1) & 1, status)) { ok = false; break; }
                 if (!mbar_wait(p_ready(b), (j >> 1) & 1, status)) { ok = false; break; }
                 tc_fence_after();
                 {   // O (+)= P V_j : M 128, N = DH, K = 64 keys; P from TMEM (8 packed columns per 16 keys),
@@ -163,10 +185,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     }
                 }
                 umma_commit(o_done);
-                umma_commit(kv_empty(b));
-                if (j + 2 < nb) {
-                    if (!mbar_wait(kv_empty(b), (j >> 1) & 1, status)) { ok = false; break; }
-                    load_kv(j + 2);
+                umma_commit(v_empty(b));
+                if (j >= 1 && j + 1 < nb) {  // value tile j-1 was consumed an iteration ago: fetch tile j+1 into its place
+                    if (!mbar_wait(v_empty(b ^ 1), ((j - 1) >> 1) & 1, status)) { ok = false; break; }
+                    load_v(j + 1);
                 }
             }
             if (!ok) *failed = 1;
@@ -304,14 +326,15 @@ cudaError_t launch_attention_tc(const CUtensorMap& tmap_q, const CUtensorMap& tm
                                 int batch, int max_seqlen, int n_heads, int n_kv_heads, int head_dim, void* out,
                                 int* status, cudaStream_t stream) {
     if (batch <= 0 || max_seqlen <= 0) return cudaSuccess;
-    const dim3 grid((max_seqlen + TC_BM - 1) / TC_BM, n_heads, batch);
+    const int n_qblocks = (max_seqlen + TC_BM - 1) / TC_BM;
+    const dim3 grid(static_cast<unsigned>(n_qblocks) * n_heads * batch);
     __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out);
     if (head_dim == 64)
-        attn_tc_kernel<64><<<grid, TC_THREADS, TcSmem<64>::TOTAL, stream>>>(tmap_q, tmap_kv, cu_seqlens_dev, n_heads,
-                                                                           n_kv_heads, o, status);
+        attn_tc_kernel<64><<<grid, TC_THREADS, TcSmem<64>::TOTAL, stream>>>(tmap_q, tmap_kv, cu_seqlens_dev, batch,
+                                                                           n_qblocks, n_heads, n_kv_heads, o, status);
     else if (head_dim == 128)
-        attn_tc_kernel<128><<<grid, TC_THREADS, TcSmem<128>::TOTAL, stream>>>(tmap_q, tmap_kv, cu_seqlens_dev, n_heads,
-                                                                             n_kv_heads, o, status);
+        attn_tc_kernel<128><<<grid, TC_THREADS, TcSmem<128>::TOTAL, stream>>>(tmap_q, tmap_kv, cu_seqlens_dev, batch,
+                                                                             n_qblocks, n_heads, n_kv_heads, o, status);
     else
         return cudaErrorInvalidValue;
     return cudaGetLastError();
