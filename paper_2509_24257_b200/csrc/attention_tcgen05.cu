@@ -100,7 +100,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         mbar_init(q_full, 1);
         mbar_init(o_done, 1);
         for (int b = 0; b < 2; ++b) {
-            mbar_init(p_ready(b), 128);
+            mbar_init(p_ready(b), 4);  // one arrival per softmax warp
             mbar_init(s_full(b), 1);
             mbar_init(v_full(b), 1);
             mbar_init(v_empty(b), 1);
@@ -265,7 +265,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             tmem_st32(s_addr, pk);
             tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(p_ready(b));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_ready(b));  // 32 arrivals on one barrier word would serialise
         }
         // The last P V must have landed before O is read.  A parity wait can only tell apart the current
         // phase and the one before it, and so far only P V_{nb-3} is known to be complete (Q K^T of the last
