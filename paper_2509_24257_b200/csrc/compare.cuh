@@ -28,11 +28,13 @@ struct CmpAcc {
     }
 
     // h: recomputed value (fp32); c_bits: committed value as a float32 bit pattern (a bf16 value widened
-    // by 16 zero bits, or the float32 itself).
+    // by 16 zero bits, or the float32 itself).  kBf16 selects the commit dtype at compile time.
+    template <bool kBf16>
     __device__ __forceinline__ void add(float h, uint32_t c_bits, const CmpParams& p) {
         const float c = __uint_as_float(c_bits);
+        const uint32_t h_bits = __float_as_uint(h);
         // finite <=> exponent field below 255
-        if (((__float_as_uint(h) >> 23) & 0xFFu) == 0xFFu || ((c_bits >> 23) & 0xFFu) == 0xFFu) {
+        if ((h_bits & 0x7F800000u) == 0x7F800000u || (c_bits & 0x7F800000u) == 0x7F800000u) {
             n_nonfinite++;
             return;
         }
@@ -47,33 +49,26 @@ struct CmpAcc {
         n_zlarge += (ad > p.tau_large) ? 1u : 0u;
 
         // both values in the commit dtype, then sign / exponent field / mantissa field
-        uint32_t hb, cb;
-        int mshift, mbits;
-        if (p.commit_dtype == VERILLM_BF16) {
+        constexpr int mshift = kBf16 ? 16 : 0;
+        constexpr int mbits = kBf16 ? 7 : 23;
+        uint32_t hb;
+        if constexpr (kBf16) {
             const __nv_bfloat16 hr = __float2bfloat16_rn(h);
             hb = static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(&hr)) << 16;
-            cb = c_bits;
-            mshift = 16;
-            mbits = 7;
         } else {
-            hb = __float_as_uint(h);
-            cb = c_bits;
-            mshift = 0;
-            mbits = 23;
+            hb = h_bits;
         }
-        const uint32_t eh = (hb >> 23) & 0xFFu, ec = (cb >> 23) & 0xFFu;
-        const int mh = static_cast<int>((hb & 0x7FFFFFu) >> mshift), mc = static_cast<int>((cb & 0x7FFFFFu) >> mshift);
+        const uint32_t cb = c_bits;
+        const uint32_t eh = hb & 0x7F800000u, ec = cb & 0x7F800000u;  // exponent fields, in place
+        const uint32_t mh = (hb & 0x7FFFFFu) >> mshift, mc = (cb & 0x7FFFFFu) >> mshift;
         if (eh != ec) {
             n_mis++;
-            const int dm = mh > mc ? mh - mc : mc - mh;
-            n_large_m += (dm > p.e_m) ? 1u : 0u;
+            n_large_m += (__usad(mh, mc, 0u) > static_cast<uint32_t>(p.e_m)) ? 1u : 0u;
         } else {
             // signed significands (implicit one unless the exponent field is zero), distance in steps
-            const int one = 1 << mbits;
-            int sh = (eh != 0u ? one : 0) + mh, sc = (ec != 0u ? one : 0) + mc;
-            if (hb >> 31) sh = -sh;
-            if (cb >> 31) sc = -sc;
-            const int dev = sh > sc ? sh - sc : sc - sh;
+            const uint32_t one = eh != 0u ? (1u << mbits) : 0u;
+            const uint32_t sh = one + mh, sc = one + mc;
+            const uint32_t dev = ((hb ^ cb) >> 31) ? sh + sc : __usad(sh, sc, 0u);
             n_small_w += (static_cast<float>(dev) <= p.thr_w) ? 1u : 0u;
             n_exact += (hb == cb) ? 1u : 0u;
         }

@@ -106,14 +106,14 @@ __global__ void compare_rows_kernel(const float* __restrict__ hidden, const void
             const uint4 cv = __ldg(c4 + j / 8);
             const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
             const float4 h1 = __ldg(reinterpret_cast<const float4*>(h + j + 4));
-            a.add(h0.x, cv.x << 16, cmp);
-            a.add(h0.y, cv.x & 0xFFFF0000u, cmp);
-            a.add(h0.z, cv.y << 16, cmp);
-            a.add(h0.w, cv.y & 0xFFFF0000u, cmp);
-            a.add(h1.x, cv.z << 16, cmp);
-            a.add(h1.y, cv.z & 0xFFFF0000u, cmp);
-            a.add(h1.z, cv.w << 16, cmp);
-            a.add(h1.w, cv.w & 0xFFFF0000u, cmp);
+            a.add<true>(h0.x, cv.x << 16, cmp);
+            a.add<true>(h0.y, cv.x & 0xFFFF0000u, cmp);
+            a.add<true>(h0.z, cv.y << 16, cmp);
+            a.add<true>(h0.w, cv.y & 0xFFFF0000u, cmp);
+            a.add<true>(h1.x, cv.z << 16, cmp);
+            a.add<true>(h1.y, cv.z & 0xFFFF0000u, cmp);
+            a.add<true>(h1.z, cv.w << 16, cmp);
+            a.add<true>(h1.w, cv.w & 0xFFFF0000u, cmp);
         }
     } else {
         const uint4* c4 =
@@ -121,10 +121,10 @@ __global__ void compare_rows_kernel(const float* __restrict__ hidden, const void
         for (int j = lane * 4; j < d; j += 128) {
             const uint4 cv = __ldg(c4 + j / 4);
             const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
-            a.add(h0.x, cv.x, cmp);
-            a.add(h0.y, cv.y, cmp);
-            a.add(h0.z, cv.z, cmp);
-            a.add(h0.w, cv.w, cmp);
+            a.add<false>(h0.x, cv.x, cmp);
+            a.add<false>(h0.y, cv.y, cmp);
+            a.add<false>(h0.z, cv.z, cmp);
+            a.add<false>(h0.w, cv.w, cmp);
         }
     }
     a.ss = warp_sum(a.ss);
@@ -205,23 +205,28 @@ __global__ void verdict_kernel(const float* __restrict__ partials, int n_layers,
     }
 }
 
-// One warp per sequence, lanes over check slots: accept iff all its checked positions were accepted (one
-// deviation above tolerance suffices to fail); score = mean MAE over its (slot, layer) cells.  Per-lane
-// double sums are combined in a fixed shuffle order, so the result is reproducible.
-__global__ void seq_verdict_kernel(const float* __restrict__ stats, const uint8_t* __restrict__ pos_ok,
-                                   const int* __restrict__ seq_of_slot, int n_check, int n_layers, int batch,
-                                   uint8_t* __restrict__ seq_ok, float* __restrict__ seq_score) {
-    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (b >= batch) return;
-    int bad = 0;
+// One block per sequence, threads over check slots: accept iff all its checked positions were accepted (one
+// deviation above tolerance suffices to fail); score = mean MAE over its (slot, layer) cells.  Per-thread
+// double sums are combined by a fixed shuffle tree and then in warp order, so the result is reproducible.
+constexpr int kSeqThreads = 256;
+__global__ void __launch_bounds__(kSeqThreads)
+seq_verdict_kernel(const float* __restrict__ stats, const uint8_t* __restrict__ pos_ok,
+                   const int* __restrict__ seq_of_slot, int n_check, int n_layers, int batch,
+                   uint8_t* __restrict__ seq_ok, float* __restrict__ seq_score) {
+    const int b = blockIdx.x;
+    int bad = 0, cells = 0;
     double sum = 0.0;
-    int cells = 0;
-    for (int s = lane; s < n_check; s += 32) {
+    for (int s = threadIdx.x; s < n_check; s += kSeqThreads) {
         if (seq_of_slot[s] != b) continue;
         bad |= (pos_ok[s] == 0) ? 1 : 0;
-        for (int l = 0; l < n_layers; ++l)
-            sum += static_cast<double>(stats[(static_cast<size_t>(s) * n_layers + l) * VERILLM_NSTAT + VERILLM_STAT_MAE]);
+        const float* mae = stats + static_cast<size_t>(s) * n_layers * VERILLM_NSTAT + VERILLM_STAT_MAE;
+        float part = 0.f;
+        int l = 0;
+        for (; l + 4 <= n_layers; l += 4)  // four independent loads in flight
+            part += (mae[(l + 0) * VERILLM_NSTAT] + mae[(l + 1) * VERILLM_NSTAT]) +
+                    (mae[(l + 2) * VERILLM_NSTAT] + mae[(l + 3) * VERILLM_NSTAT]);
+        for (; l < n_layers; ++l) part += mae[l * VERILLM_NSTAT];
+        sum += static_cast<double>(part);
         cells += n_layers;
     }
 #pragma unroll
@@ -230,9 +235,24 @@ __global__ void seq_verdict_kernel(const float* __restrict__ stats, const uint8_
         sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
         cells += __shfl_xor_sync(0xFFFFFFFFu, cells, o);
     }
-    if (lane == 0) {
-        seq_ok[b] = bad ? 0 : 1;
-        seq_score[b] = cells > 0 ? static_cast<float>(sum / static_cast<double>(cells)) : 0.f;
+    __shared__ double w_sum[kSeqThreads / 32];
+    __shared__ int w_bad[kSeqThreads / 32], w_cells[kSeqThreads / 32];
+    if ((threadIdx.x & 31) == 0) {
+        w_sum[threadIdx.x >> 5] = sum;
+        w_bad[threadIdx.x >> 5] = bad;
+        w_cells[threadIdx.x >> 5] = cells;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        int bd = 0, c = 0;
+        for (int w = 0; w < kSeqThreads / 32; ++w) {
+            t += w_sum[w];
+            bd |= w_bad[w];
+            c += w_cells[w];
+        }
+        seq_ok[b] = bd ? 0 : 1;
+        seq_score[b] = c > 0 ? static_cast<float>(t / static_cast<double>(c)) : 0.f;
     }
 }
 
@@ -514,7 +534,7 @@ cudaError_t launch_verdict(const float* partials, int n_layers, int n_check, int
 cudaError_t launch_seq_verdict(const float* stats, const uint8_t* pos_ok, const int* seq_of_slot, int n_check,
                                int n_layers, int batch, uint8_t* seq_ok, float* seq_score, cudaStream_t s) {
     if (batch <= 0) return cudaSuccess;
-    seq_verdict_kernel<<<(batch + 3) / 4, 128, 0, s>>>(stats, pos_ok, seq_of_slot, n_check, n_layers, batch, seq_ok,
+    seq_verdict_kernel<<<batch, kSeqThreads, 0, s>>>(stats, pos_ok, seq_of_slot, n_check, n_layers, batch, seq_ok,
                                                         seq_score);
     return cudaGetLastError();
 }

@@ -230,14 +230,14 @@ __device__ __forceinline__ void compare_row(const GemmParams& p, int row, int n0
                 const uint4 cv = __ldg(c4 + j / 8);
                 const float4 h0 = *reinterpret_cast<const float4*>(hrow + j);
                 const float4 h1 = *reinterpret_cast<const float4*>(hrow + j + 4);
-                acc.add(h0.x, cv.x << 16, p.cmp);
-                acc.add(h0.y, cv.x & 0xFFFF0000u, p.cmp);
-                acc.add(h0.z, cv.y << 16, p.cmp);
-                acc.add(h0.w, cv.y & 0xFFFF0000u, p.cmp);
-                acc.add(h1.x, cv.z << 16, p.cmp);
-                acc.add(h1.y, cv.z & 0xFFFF0000u, p.cmp);
-                acc.add(h1.z, cv.w << 16, p.cmp);
-                acc.add(h1.w, cv.w & 0xFFFF0000u, p.cmp);
+                acc.add<true>(h0.x, cv.x << 16, p.cmp);
+                acc.add<true>(h0.y, cv.x & 0xFFFF0000u, p.cmp);
+                acc.add<true>(h0.z, cv.y << 16, p.cmp);
+                acc.add<true>(h0.w, cv.y & 0xFFFF0000u, p.cmp);
+                acc.add<true>(h1.x, cv.z << 16, p.cmp);
+                acc.add<true>(h1.y, cv.z & 0xFFFF0000u, p.cmp);
+                acc.add<true>(h1.z, cv.w << 16, p.cmp);
+                acc.add<true>(h1.w, cv.w & 0xFFFF0000u, p.cmp);
                 if (hout) {
                     *reinterpret_cast<float4*>(hout + j) = h0;
                     *reinterpret_cast<float4*>(hout + j + 4) = h1;
@@ -250,10 +250,10 @@ __device__ __forceinline__ void compare_row(const GemmParams& p, int row, int n0
             for (int j = 0; j < ncols; j += 4) {
                 const uint4 cv = __ldg(c4 + j / 4);
                 const float4 h0 = *reinterpret_cast<const float4*>(hrow + j);
-                acc.add(h0.x, cv.x, p.cmp);
-                acc.add(h0.y, cv.y, p.cmp);
-                acc.add(h0.z, cv.z, p.cmp);
-                acc.add(h0.w, cv.w, p.cmp);
+                acc.add<false>(h0.x, cv.x, p.cmp);
+                acc.add<false>(h0.y, cv.y, p.cmp);
+                acc.add<false>(h0.z, cv.z, p.cmp);
+                acc.add<false>(h0.w, cv.w, p.cmp);
                 if (hout) *reinterpret_cast<float4*>(hout + j) = h0;
             }
         }

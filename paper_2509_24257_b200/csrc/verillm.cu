@@ -503,6 +503,7 @@ static int verify_impl(verillm_model* m, const int32_t* tokens, const void* stat
                        const int32_t* check_seq, const int32_t* check_pos, int32_t n_check, const verillm_tol* tol,
                        const verillm_report* rep, void* cuda_stream) {
     if (!m || (!tokens && !states_in) || !tol || !rep) return VERILLM_E_INVAL;
+    if (tol->e_m < 0 || !(tol->e_w >= 0.f)) return VERILLM_E_INVAL;
     if (l0 < 0 || l1 > m->cfg.n_layers || l0 >= l1) return VERILLM_E_RANGE;
     if (commit_dtype != VERILLM_BF16 && commit_dtype != VERILLM_F32) return VERILLM_E_INVAL;
     if (!rep->seq_ok || !rep->seq_score || !rep->status) return VERILLM_E_INVAL;
@@ -578,6 +579,7 @@ int verillm_compare(const float* hidden, const void* committed, int32_t commit_d
                     int32_t d_model, const int32_t* check_seq, int32_t batch, const verillm_tol* tol,
                     const verillm_report* rep, void* cuda_stream) {
     if (!hidden || !committed || !check_seq || !tol || !rep) return VERILLM_E_INVAL;
+    if (tol->e_m < 0 || !(tol->e_w >= 0.f)) return VERILLM_E_INVAL;
     if (commit_dtype != VERILLM_BF16 && commit_dtype != VERILLM_F32) return VERILLM_E_INVAL;
     if (n_layers < 1 || n_check < 1 || batch < 1) return VERILLM_E_INVAL;
     if (d_model < 8 || d_model % 8 != 0) return VERILLM_E_SHAPE;
@@ -619,6 +621,7 @@ int verillm_compare_noalloc(const float* hidden, const void* committed, int32_t 
                             int32_t n_check, int32_t d_model, const int32_t* check_seq, int32_t batch,
                             const verillm_tol* tol, const verillm_report* rep, void* cuda_stream) {
     if (!hidden || !committed || !check_seq || !tol || !rep) return VERILLM_E_INVAL;
+    if (tol->e_m < 0 || !(tol->e_w >= 0.f)) return VERILLM_E_INVAL;
     if (commit_dtype != VERILLM_BF16 && commit_dtype != VERILLM_F32) return VERILLM_E_INVAL;
     if (n_layers < 1 || n_check < 1 || batch < 1) return VERILLM_E_INVAL;
     if (d_model < 8 || d_model % 8 != 0) return VERILLM_E_SHAPE;
