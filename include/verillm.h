@@ -226,6 +226,25 @@ int verillm_compare_noalloc(const float *hidden, const void *committed, int32_t 
                             int32_t n_check, int32_t d_model, const int32_t *check_seq, int32_t batch,
                             const verillm_tol *tol, const verillm_report *report, void *cuda_stream);
 
+/* Relaxed spot check on sampled scalar entries (the on-chain value matching: Delta_j = |v_j - V_j| <= eps,
+ * agreement rate p_hat = (1/n) sum 1[Delta_j <= eps], positive verdict iff p_hat >= theta).
+ *  hidden      DEVICE float32 [n_rows][d_model]: the verifier's states (e.g. one layer of hidden_out)
+ *  sample_row / sample_col  HOST int32 [n_samples]: the sampled entries; reference HOST float32 [n_samples]: V_j
+ *  agree_out   DEVICE uint8 [n_samples]; p_hat_out DEVICE float [1]; verdict_out DEVICE uint8 [1]
+ * The comparison is made in float32; a NaN never agrees.  Staging memory comes from the stream-ordered
+ * allocator.  Errors: E_INVAL, E_RANGE (an index outside the matrix). */
+int verillm_spot_check(const float *hidden, int32_t n_rows, int32_t d_model, const int32_t *sample_row,
+                       const int32_t *sample_col, const float *reference, int32_t n_samples, float eps, float theta,
+                       uint8_t *agree_out, float *p_hat_out, uint8_t *verdict_out, void *cuda_stream);
+
+/* Merkle commitment of hidden states ("serializes its output tensor, constructs a Merkle tree over all scalar
+ * entries and submits the Merkle root"; canonical float32 leaves, SHA-256): one root per vector.
+ *  states    DEVICE float32 [n_vec][d_model]; roots_out DEVICE uint8 [n_vec][32]
+ * Leaf j = SHA-256(4 bytes of entry j, little-endian IEEE-754 float32); node = SHA-256(left || right); an odd
+ * node at the end of a level is paired with itself; a single entry's leaf is its own root.
+ * Errors: E_INVAL, E_SHAPE (d_model > 12800), E_ARCH, E_CUDA. */
+int verillm_merkle_roots(const float *states, int32_t n_vec, int32_t d_model, uint8_t *roots_out, void *cuda_stream);
+
 /* Single steps of the path, exposed for testing against the oracle.  All pointers DEVICE. */
 
 /* C[M][N] = A[M][K] * B[N][K]^T, bf16 inputs, fp32 accumulation on the tensor cores; out_f32 selects a

@@ -433,6 +433,48 @@ def verify_segment(
     return Report(stats, pos_ok, first_bad, seq_ok, seq_score, hidden)
 
 
+def merkle_root(vec: np.ndarray) -> bytes:
+    """Merkle root of one hidden-state vector: leaves are SHA-256 of each entry's canonical float32 serialisation
+    (4 bytes, little endian), inner nodes SHA-256(left || right); a level with an odd number of nodes pairs its
+    last node with itself; a single leaf is its own root."""
+    import hashlib
+    import struct
+
+    level = [hashlib.sha256(struct.pack("<f", float(np.float32(x)))).digest() for x in np.asarray(vec).reshape(-1)]
+    while len(level) > 1:
+        if len(level) % 2:
+            level.append(level[-1])
+        level = [hashlib.sha256(level[i] + level[i + 1]).digest() for i in range(0, len(level), 2)]
+    return level[0]
+
+
+def merkle_path(vec: np.ndarray, index: int):
+    """Inclusion proof of leaf `index`: the sibling digests from the leaf level up."""
+    import hashlib
+    import struct
+
+    level = [hashlib.sha256(struct.pack("<f", float(np.float32(x)))).digest() for x in np.asarray(vec).reshape(-1)]
+    path = []
+    while len(level) > 1:
+        if len(level) % 2:
+            level.append(level[-1])
+        path.append(level[index ^ 1])
+        level = [hashlib.sha256(level[i] + level[i + 1]).digest() for i in range(0, len(level), 2)]
+        index //= 2
+    return path
+
+
+def spot_check(hidden: np.ndarray, sample_row, sample_col, reference, eps: float, theta: float):
+    """Relaxed on-chain test on sampled scalars: Delta_j = |v_j - V_j| <= eps, p_hat = mean 1[Delta_j <= eps],
+    verdict = p_hat >= theta.  The threshold decision is taken on float32 values, the precision in which the
+    entries are serialised.  Returns (agree [n] uint8, p_hat, verdict)."""
+    v = np.asarray(hidden)[np.asarray(sample_row), np.asarray(sample_col)].astype(np.float32)
+    with np.errstate(invalid="ignore"):
+        agree = np.abs(v - np.asarray(reference, dtype=np.float32)) <= np.float32(eps)
+    p_hat = float(np.float32(agree.sum()) / np.float32(len(agree)))
+    return agree.astype(np.uint8), p_hat, bool(np.float32(p_hat) >= np.float32(theta))
+
+
 def token_match(m: Model, last_hidden: np.ndarray, lm_head: np.ndarray, claimed: np.ndarray):
     """Tail token check: TokenMatch(argmax f_LM(S_{L+1}), y) with f_LM = output head after the final RMSNorm.
 

@@ -30,7 +30,7 @@ EXPORTS = (
     "verillm_verify_prefill", "verillm_decode_commit", "verillm_compare", "verillm_compare_noalloc", "verillm_op_gemm",
     "verillm_op_rmsnorm", "verillm_op_attention", "verillm_free", "verillm_strerror",
     "verillm_last_launch_count", "verillm_profile_enable", "verillm_profile_read",
-    "verillm_load_lm_head", "verillm_token_match", "verillm_verify_segment",
+    "verillm_load_lm_head", "verillm_token_match", "verillm_verify_segment", "verillm_spot_check", "verillm_merkle_roots",
 )
 PROF_CLASSES = ("setup", "rmsnorm", "gemm_qkv_rope", "attention", "gemm_o_resid", "gemm_gate_up_swiglu",
                 "gemm_down_resid_compare", "verdict")
@@ -114,6 +114,11 @@ def lib() -> C.CDLL:
             C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(Tol), C.POINTER(ReportC), C.c_void_p,
         ]
         L.verillm_verify_segment.restype = C.c_int
+        L.verillm_spot_check.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                         C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.verillm_spot_check.restype = C.c_int
+        L.verillm_merkle_roots.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.verillm_merkle_roots.restype = C.c_int
         L.verillm_load_lm_head.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
         L.verillm_load_lm_head.restype = C.c_int
         L.verillm_token_match.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -386,6 +391,33 @@ def compare_noalloc(hidden: torch.Tensor, committed: torch.Tensor, check_seq: Se
                                              cs.ctypes.data, batch, C.byref(tol), C.byref(st), _stream_ptr(stream))
     _check(code, "verillm_compare_noalloc")
     return rep
+
+
+def spot_check(hidden: torch.Tensor, sample_row, sample_col, reference, eps: float, theta: float,
+               stream: Optional[torch.cuda.Stream] = None):
+    """Sampled value matching on hidden (float32 device [n_rows][d]).  Returns device (agree uint8 [n], p_hat f32 [1], ok uint8 [1])."""
+    rows, cols = _i32(sample_row), _i32(sample_col)
+    ref = np.ascontiguousarray(np.asarray(reference, dtype=np.float32))
+    n = int(rows.shape[0])
+    agree = torch.empty(n, dtype=torch.uint8, device=hidden.device)
+    p_hat = torch.empty(1, dtype=torch.float32, device=hidden.device)
+    ok = torch.empty(1, dtype=torch.uint8, device=hidden.device)
+    with torch.cuda.device(hidden.device):
+        _check(lib().verillm_spot_check(hidden.data_ptr(), hidden.shape[0], hidden.shape[1], rows.ctypes.data,
+                                        cols.ctypes.data, ref.ctypes.data, n, float(eps), float(theta), agree.data_ptr(),
+                                        p_hat.data_ptr(), ok.data_ptr(), _stream_ptr(stream)), "verillm_spot_check")
+    return agree, p_hat, ok
+
+
+def merkle_roots(states: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """states float32 device [n_vec][d] -> uint8 device [n_vec][32] SHA-256 Merkle roots over float32 leaves."""
+    if states.dtype != torch.float32 or not states.is_contiguous() or states.dim() != 2:
+        raise ValueError("states must be a contiguous float32 matrix")
+    roots = torch.empty(states.shape[0], 32, dtype=torch.uint8, device=states.device)
+    with torch.cuda.device(states.device):
+        _check(lib().verillm_merkle_roots(states.data_ptr(), states.shape[0], states.shape[1], roots.data_ptr(),
+                                          _stream_ptr(stream)), "verillm_merkle_roots")
+    return roots
 
 
 def op_gemm(a: torch.Tensor, b: torch.Tensor, out_f32: bool = False) -> torch.Tensor:

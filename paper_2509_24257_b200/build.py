@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libverillm.so")
-SOURCES = ["gemm_tcgen05.cu", "attention_tcgen05.cu", "elementwise.cu", "verillm.cu"]
+SOURCES = ["gemm_tcgen05.cu", "attention_tcgen05.cu", "elementwise.cu", "merkle.cu", "verillm.cu"]
 HEADERS = ["common.cuh", "compare.cuh", "kernels.h", os.path.join("..", "..", "include", "verillm.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -298,6 +298,32 @@ __global__ void argmax_reduce_kernel(const float4* __restrict__ records, int row
     }
 }
 
+// ------------------------------------------------------------------ sampled value matching
+// One block: threads stride over the samples, agreement counts are integers, so the reduction order is free.
+__global__ void __launch_bounds__(256)
+spot_check_kernel(const float* __restrict__ hidden, int d, const int* __restrict__ rows, const int* __restrict__ cols,
+                  const float* __restrict__ ref, int n, float eps, float theta, uint8_t* __restrict__ agree,
+                  float* __restrict__ p_hat, uint8_t* __restrict__ ok) {
+    uint32_t cnt = 0;
+    for (int j = threadIdx.x; j < n; j += blockDim.x) {
+        const float v = hidden[static_cast<size_t>(rows[j]) * d + cols[j]];
+        const bool a = fabsf(v - ref[j]) <= eps;  // false for NaN
+        agree[j] = a ? 1 : 0;
+        cnt += a ? 1u : 0u;
+    }
+    __shared__ uint32_t part[8];
+    cnt = warp_sum_u32(cnt);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = cnt;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t t = 0;
+        for (int w = 0; w < 8; ++w) t += part[w];
+        const float p = static_cast<float>(t) / static_cast<float>(n);
+        *p_hat = p;
+        *ok = p >= theta ? 1 : 0;
+    }
+}
+
 // ------------------------------------------------------------------ decode-side kernels
 // out[r][n] (+)= sum_k x[r][k] * w[n][k] for up to 8 rows: one warp per output column streams the
 // weight row once (16-byte loads) and keeps one accumulator per row.
@@ -544,6 +570,13 @@ cudaError_t launch_argmax_reduce(const float* records, int rows, int n_tiles, co
     if (rows <= 0) return cudaSuccess;
     argmax_reduce_kernel<<<(rows + 3) / 4, 128, 0, s>>>(reinterpret_cast<const float4*>(records), rows, n_tiles, claimed,
                                                        argmax_out, match_out, margin_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_spot_check(const float* hidden, int d, const int* rows, const int* cols, const float* ref, int n,
+                              float eps, float theta, uint8_t* agree, float* p_hat, uint8_t* ok, cudaStream_t s) {
+    if (n <= 0) return cudaErrorInvalidValue;
+    spot_check_kernel<<<1, 256, 0, s>>>(hidden, d, rows, cols, ref, n, eps, theta, agree, p_hat, ok);
     return cudaGetLastError();
 }
 

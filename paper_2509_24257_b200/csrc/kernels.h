@@ -90,6 +90,14 @@ cudaError_t launch_seq_verdict(const float* stats, const uint8_t* pos_ok, const 
 cudaError_t launch_argmax_reduce(const float* records, int rows, int n_tiles, const int* claimed, int* argmax_out,
                                  uint8_t* match_out, float* margin_out, cudaStream_t stream);
 
+// Sampled value matching: agree[j] = |hidden[row_j][col_j] - ref_j| <= eps; p_hat = mean(agree); ok = p_hat >= theta.
+cudaError_t launch_spot_check(const float* hidden, int d, const int* rows, const int* cols, const float* ref, int n,
+                              float eps, float theta, uint8_t* agree, float* p_hat, uint8_t* ok, cudaStream_t stream);
+
+// Merkle roots (SHA-256 over little-endian float32 leaves), one 32-byte root per vector of d entries.
+cudaError_t merkle_init();  // derives the SHA-256 constants and uploads them (once per device)
+cudaError_t launch_merkle_roots(const float* states, int n_vec, int d, uint8_t* roots, cudaStream_t stream);
+
 // ------------------------------------------------------------------ decode (prover side)
 // out[rows][n] (fp32) = x[rows][k] (bf16) * w[n][k]^T, rows <= 8 per launch group; optional in-place add.
 cudaError_t launch_skinny_gemm(const void* x, const void* w, float* out, int rows, int n, int k, int accumulate,

@@ -110,6 +110,7 @@ int ensure_init() {
     if (prop.major != 10) return VERILLM_E_ARCH;
     CU_TRY(gemm_init());
     CU_TRY(attention_tc_init());
+    CU_TRY(merkle_init());
     done[dev] = true;
     return VERILLM_OK;
 }
@@ -693,6 +694,37 @@ int verillm_token_match(verillm_model* m, const float* last_hidden, const int32_
     CU_TRY(cudaMemsetAsync(m->status, 0, sizeof(int), st));
     CU_TRY(launch_gemm(EPI_ARGMAX, m->t_tm_y, p.pair ? m->t_lm_h : m->t_lm, p, m->num_sms, st));
     CU_TRY(launch_argmax_reduce(m->tm_rec, n_check, m->n_tiles_v, m->tm_claimed, argmax_out, match_out, margin_out, st));
+    return VERILLM_OK;
+}
+
+int verillm_spot_check(const float* hidden, int32_t n_rows, int32_t d_model, const int32_t* sample_row,
+                       const int32_t* sample_col, const float* reference, int32_t n_samples, float eps, float theta,
+                       uint8_t* agree_out, float* p_hat_out, uint8_t* verdict_out, void* cuda_stream) {
+    if (!hidden || !sample_row || !sample_col || !reference || !agree_out || !p_hat_out || !verdict_out) return VERILLM_E_INVAL;
+    if (n_rows < 1 || d_model < 1 || n_samples < 1 || !(eps >= 0.f)) return VERILLM_E_INVAL;
+    for (int j = 0; j < n_samples; ++j)
+        if (sample_row[j] < 0 || sample_row[j] >= n_rows || sample_col[j] < 0 || sample_col[j] >= d_model) return VERILLM_E_RANGE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    char* buf = nullptr;
+    const size_t n = static_cast<size_t>(n_samples);
+    CU_TRY(cudaMallocAsync(reinterpret_cast<void**>(&buf), n * 12, st));
+    int* rows = reinterpret_cast<int*>(buf);
+    int* cols = rows + n;
+    float* ref = reinterpret_cast<float*>(cols + n);
+    CU_TRY(cudaMemcpyAsync(rows, sample_row, n * 4, cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(cols, sample_col, n * 4, cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(ref, reference, n * 4, cudaMemcpyHostToDevice, st));
+    CU_TRY(launch_spot_check(hidden, d_model, rows, cols, ref, n_samples, eps, theta, agree_out, p_hat_out, verdict_out, st));
+    CU_TRY(cudaFreeAsync(buf, st));
+    return VERILLM_OK;
+}
+
+int verillm_merkle_roots(const float* states, int32_t n_vec, int32_t d_model, uint8_t* roots_out, void* cuda_stream) {
+    if (!states || !roots_out || n_vec < 1 || d_model < 1) return VERILLM_E_INVAL;
+    if (d_model > 12800) return VERILLM_E_SHAPE;  // one level of the tree must fit in shared memory
+    int rc = ensure_init();
+    if (rc) return rc;
+    CU_TRY(launch_merkle_roots(states, n_vec, d_model, roots_out, reinterpret_cast<cudaStream_t>(cuda_stream)));
     return VERILLM_OK;
 }
 

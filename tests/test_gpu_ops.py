@@ -156,3 +156,35 @@ def test_tensor_core_kernels_are_bit_reproducible_over_many_launches():
     ref = vb.op_gemm(a, b)
     for _ in range(300):
         assert torch.equal(vb.op_gemm(a, b), ref)
+
+
+def test_spot_check_matches_oracle_bit_for_bit():
+    rng = np.random.default_rng(31)
+    hidden = rng.standard_normal((82, 4096)).astype(np.float32)
+    n = 3584  # the largest sample count in the paper's tables
+    rows, cols = rng.integers(0, 82, n), rng.integers(0, 4096, n)
+    ref = hidden[rows, cols] + (rng.standard_normal(n) * 0.01).astype(np.float32)
+    ref[::97] = np.nan
+    for eps, theta in ((0.01, 0.6), (0.02, 0.99), (0.0, 0.0)):
+        agree_o, p_o, ok_o = vo.spot_check(hidden, rows, cols, ref, eps, theta)
+        agree, p_hat, ok = vb.spot_check(torch.from_numpy(hidden).to(DEV), rows, cols, ref, eps, theta)
+        assert np.array_equal(agree.cpu().numpy(), agree_o)
+        assert float(p_hat.item()) == np.float32(p_o) and bool(ok.item()) == ok_o
+    with pytest.raises(vb.VerillmError) as e:
+        vb.spot_check(torch.from_numpy(hidden).to(DEV), [82], [0], [0.0], 0.1, 0.5)
+    assert e.value.code == vb.E_RANGE
+
+
+@pytest.mark.parametrize("n_vec,d", [(5, 1), (7, 2), (3, 3), (4, 257), (6, 1024), (3, 4096), (2, 8192), (2, 5000)])
+def test_merkle_roots_are_bit_exact(n_vec, d):
+    rng = np.random.default_rng(100 + d)
+    x = rng.standard_normal((n_vec, d)).astype(np.float32)
+    x[0, 0] = -0.0
+    if d > 2:
+        x[-1, 1], x[-1, 2] = np.inf, np.nan  # every bit pattern is just four bytes to the hash
+    roots = vb.merkle_roots(torch.from_numpy(x).to(DEV)).cpu().numpy()
+    for i in range(n_vec):
+        assert roots[i].tobytes() == vo.merkle_root(x[i]), (i, d)
+    with pytest.raises(vb.VerillmError) as e:
+        vb.merkle_roots(torch.zeros(1, 12801, device=DEV))
+    assert e.value.code == vb.E_SHAPE

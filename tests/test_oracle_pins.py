@@ -437,3 +437,52 @@ def test_segments_compose_to_the_full_pass():
     assert rep.pos_ok[2] == 0 and rel[2] > 0.1  # the perturbed position itself
     assert rel[1] < 1e-6  # another sequence: untouched
     assert 1e-6 < rel[0] < rel[2]  # a later position of the same sequence attends to it and moves, but less
+
+
+def test_spot_check_worked_example():
+    """Eight sampled scalars, tolerance 0.01: worked by hand."""
+    hidden = np.arange(12, dtype=np.float64).reshape(3, 4) / 8.0
+    rows, cols = [0, 0, 1, 1, 2, 2, 2, 0], [0, 3, 1, 2, 0, 3, 1, 1]
+    ref = hidden[rows, cols].copy()
+    ref[1] += 0.01      # exactly at the tolerance: agrees (<=)
+    ref[2] -= 0.0101    # just beyond: disagrees
+    ref[5] = np.nan     # never agrees
+    ref[7] += 1.0
+    agree, p_hat, ok = vo.spot_check(hidden, rows, cols, ref, 0.01, 0.625)
+    assert agree.tolist() == [1, 1, 0, 1, 1, 0, 1, 0] and p_hat == 5 / 8 and ok  # 0.625 >= theta
+    assert not vo.spot_check(hidden, rows, cols, ref, 0.01, 0.63)[2]
+
+
+def test_merkle_root_structure_and_inclusion_proofs():
+    """The tree against an independent verifier that only knows 'hash the leaf, then fold the path'."""
+    import hashlib
+    import struct
+
+    def verify(root, value, index, path):  # MerkleVerify as a contract would run it
+        h = hashlib.sha256(struct.pack("<f", value)).digest()
+        for sib in path:
+            h = hashlib.sha256(sib + h).digest() if index & 1 else hashlib.sha256(h + sib).digest()
+            index >>= 1
+        return h == root
+
+    rng = np.random.default_rng(41)
+    for n in (1, 2, 3, 5, 8, 13, 64):
+        v = rng.standard_normal(n).astype(np.float32)
+        root = vo.merkle_root(v)
+        assert len(root) == 32
+        for j in range(n):
+            path = vo.merkle_path(v, j)
+            assert len(path) == int(np.ceil(np.log2(n))) if n > 1 else path == []
+            assert verify(root, float(v[j]), j, path)
+            assert not verify(root, float(v[j]) + 1.0, j, path)
+        w = v.copy()
+        w[n // 2] = np.nextafter(w[n // 2], np.float32(10.0))  # one ulp in one leaf
+        assert vo.merkle_root(w) != root
+    # serialisation: float32 little endian, so -0.0 and 0.0 commit differently and float64 input is narrowed first
+    assert vo.merkle_root(np.array([0.0])) == hashlib.sha256(bytes(4)).digest()
+    assert vo.merkle_root(np.array([-0.0])) == hashlib.sha256(bytes.fromhex("00000080")).digest()
+    assert vo.merkle_root(np.array([1.0])) == hashlib.sha256(bytes.fromhex("0000803f")).digest()
+    assert vo.merkle_root(np.array([0.1], dtype=np.float64)) == vo.merkle_root(np.array([np.float32(0.1)]))
+    two = vo.merkle_root(np.array([1.0, 2.0]))
+    assert two == hashlib.sha256(hashlib.sha256(bytes.fromhex("0000803f")).digest()
+                                 + hashlib.sha256(bytes.fromhex("00000040")).digest()).digest()
