@@ -376,6 +376,22 @@ def run_ours(args, wl):
                     "frac": round(cmp_bytes / (cmp_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
     del hid, com
 
+    # ---- Merkle commitment of the checked states (one SHA-256 tree per (layer, position) vector): integer ALU work
+    mk_in = torch.randn(s.n_layers * len(cs), s.d_model, device=device)
+    vb.merkle_roots(mk_in, stream)
+    m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    m0.record(stream)
+    for _ in range(5):
+        vb.merkle_roots(mk_in, stream)
+    m1.record(stream)
+    torch.cuda.synchronize()
+    mk_ms = m0.elapsed_time(m1) / 5
+    n_compress = mk_in.shape[0] * (4 * ((s.d_model + 1) // 2) + 2 * ((s.d_model + 1) // 2 - 1))
+    merkle = {"vectors": int(mk_in.shape[0]), "scalars_per_vector": s.d_model, "ms": round(mk_ms, 4), "bound": "alu",
+              "ns_per_scalar": round(mk_ms * 1e6 / mk_in.numel(), 4),
+              "sha256_compressions_per_s": round(n_compress / (mk_ms * 1e-3), 0)}
+    del mk_in
+
     if rank == 0:
         run, desc = oracle_sample(wl, 12.0, str(device)) if args.gpus == 1 else (None, None)
         cpu_baseline = None
@@ -402,7 +418,7 @@ def run_ours(args, wl):
                          "status": res["status"]},
             "clocks": clocks, "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                                      "d2h_bytes_per_step": int(d2h)},
-            "gpu_launches": int(launches), "roofline": roofline, "token_match": token_match, "compare_path": compare_path,
+            "gpu_launches": int(launches), "roofline": roofline, "token_match": token_match, "compare_path": compare_path, "merkle": merkle,
             "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))

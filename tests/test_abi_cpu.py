@@ -46,6 +46,13 @@ def test_bad_arguments_are_rejected_on_the_host(library):
     assert library.verillm_verify_prefill(None, None, None, 1, None, 0, None, None, 0, ctypes.byref(tol), ctypes.byref(rep), None) == vb.E_INVAL
     assert library.verillm_compare(None, None, 0, 1, 1, 64, None, 1, ctypes.byref(tol), ctypes.byref(rep), None) == vb.E_INVAL
     assert library.verillm_op_gemm(None, None, None, 1, 1, 1, 0, None, None) == vb.E_INVAL
+    z = ctypes.c_void_p()
+    assert library.verillm_spot_check(None, 1, 1, None, None, None, 1, ctypes.c_float(0.1), ctypes.c_float(0.5), None, None, None, None) == vb.E_INVAL
+    assert library.verillm_merkle_roots(None, 1, 8, None, None) == vb.E_INVAL
+    assert library.verillm_token_match(None, None, None, 1, None, None, None, None) == vb.E_INVAL
+    assert library.verillm_load_lm_head(None, None, 0) == vb.E_INVAL
+    assert library.verillm_verify_segment(None, None, 0, 0, 1, None, 1, None, 0, None, None, 0, ctypes.byref(tol), ctypes.byref(rep), None) == vb.E_INVAL
+    assert library.verillm_compare_noalloc(None, None, 0, 1, 1, 64, None, 1, ctypes.byref(tol), ctypes.byref(rep), None) == vb.E_INVAL
     library.verillm_free(None)  # a no-op
 
 
