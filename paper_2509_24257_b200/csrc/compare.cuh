@@ -14,9 +14,32 @@ constexpr int kNPart = 12;
 struct CmpParams {
     int commit_dtype;  // VERILLM_BF16 / VERILLM_F32
     float tau_large;   // Z_large threshold
-    float thr_w;       // e_w * 2^mantissa_bits: largest significand distance counted as small
-    int e_m;           // mantissa-field distance above which a mismatch is large
+    // Both thresholds of the bit-aware test are integers in the units of a float32 bit pattern (a bf16
+    // mantissa field sits in bits 16..22 of the widened value, the implicit one at bit 23):
+    int thr_dev;  // largest significand distance counted as small, -1 if none qualifies
+    int thr_em;   // mantissa-field distance above which an exponent mismatch is large
 };
+
+// Host-side conversion of (e_w, e_m) to those units.  `dev <= e_w * 2^mantissa_bits` on an integer
+// distance is `dev <= floor(e_w * 2^mantissa_bits)`; distances never exceed 2^(mantissa_bits + 2).
+inline CmpParams make_cmp_params(int commit_dtype, float tau_large, float e_w, int e_m) {
+    const int mbits = commit_dtype == VERILLM_BF16 ? 7 : 23;
+    const int mshift = 23 - mbits;
+    const float thr_w = e_w * static_cast<float>(1 << mbits);
+    const int max_dev = 1 << (mbits + 2);
+    int k = -1;
+    if (thr_w >= static_cast<float>(max_dev)) k = max_dev;
+    else if (thr_w >= 0.f) k = static_cast<int>(thr_w);  // floor of a non-negative value
+    int em = e_m;
+    if (em < -1) em = -1;
+    if (em > (1 << mbits)) em = 1 << mbits;
+    CmpParams c;
+    c.commit_dtype = commit_dtype;
+    c.tau_large = tau_large;
+    c.thr_dev = k < 0 ? -1 : k * (1 << mshift);
+    c.thr_em = em * (1 << mshift);
+    return c;
+}
 
 struct CmpAcc {
     float ss, rr, sa, sg, mx;
@@ -27,19 +50,20 @@ struct CmpAcc {
         n_mis = n_large_m = n_small_w = n_exact = n_qsmall = n_zlarge = n_nonfinite = 0u;
     }
 
-    // h: recomputed value (fp32); c_bits: committed value as a float32 bit pattern (a bf16 value widened
-    // by 16 zero bits, or the float32 itself).  kBf16 selects the commit dtype at compile time.
-    template <bool kBf16>
-    __device__ __forceinline__ void add(float h, uint32_t c_bits, const CmpParams& p) {
-        const float c = __uint_as_float(c_bits);
-        const uint32_t h_bits = __float_as_uint(h);
-        // finite <=> exponent field below 255
-        if ((h_bits & 0x7F800000u) == 0x7F800000u || (c_bits & 0x7F800000u) == 0x7F800000u) {
-            n_nonfinite++;
-            return;
-        }
+    // h: recomputed value (fp32); hb: h rounded to the commit dtype, as a float32 bit pattern; cb: the
+    // committed value as a float32 bit pattern (a bf16 value widened by 16 zero bits, or the float32).
+    __device__ __forceinline__ void add_bits(float h, uint32_t hb, uint32_t cb, const CmpParams& p) {
+        const float c = __uint_as_float(cb);
         const float d = h - c;
         const float ad = fabsf(d);
+        if (!(ad < INFINITY)) {
+            // rare: a non-finite operand (counted and left out of every sum), or a finite pair whose
+            // difference overflowed (kept)
+            if ((__float_as_uint(h) & 0x7F800000u) == 0x7F800000u || (cb & 0x7F800000u) == 0x7F800000u) {
+                n_nonfinite++;
+                return;
+            }
+        }
         ss = fmaf(d, d, ss);
         rr = fmaf(c, c, rr);
         sa += ad;
@@ -48,30 +72,32 @@ struct CmpAcc {
         n_qsmall += (ad <= 1e-5f) ? 1u : 0u;
         n_zlarge += (ad > p.tau_large) ? 1u : 0u;
 
-        // both values in the commit dtype, then sign / exponent field / mantissa field
-        constexpr int mshift = kBf16 ? 16 : 0;
-        constexpr int mbits = kBf16 ? 7 : 23;
-        uint32_t hb;
-        if constexpr (kBf16) {
-            const __nv_bfloat16 hr = __float2bfloat16_rn(h);
-            hb = static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(&hr)) << 16;
-        } else {
-            hb = h_bits;
+        // sign / exponent field / mantissa field of both values in the commit dtype
+        const uint32_t x = hb ^ cb;
+        const bool same_exp = (x & 0x7F800000u) == 0u;
+        const uint32_t mh = hb & 0x7FFFFFu, mc = cb & 0x7FFFFFu;
+        int dev = static_cast<int>(__usad(mh, mc, 0u));  // mantissa-field distance; also the significand
+                                                          // distance when exponent and sign agree
+        n_mis += same_exp ? 0u : 1u;
+        n_large_m += (!same_exp && dev > p.thr_em) ? 1u : 0u;
+        if (same_exp && static_cast<int>(x) < 0) {
+            // rare: equal exponent fields, opposite signs: the signed significands (implicit one unless the
+            // exponent field is zero) lie on both sides of zero
+            const uint32_t one = (hb & 0x7F800000u) != 0u ? 0x800000u : 0u;
+            dev = static_cast<int>(mh + mc + 2u * one);
         }
-        const uint32_t cb = c_bits;
-        const uint32_t eh = hb & 0x7F800000u, ec = cb & 0x7F800000u;  // exponent fields, in place
-        const uint32_t mh = (hb & 0x7FFFFFu) >> mshift, mc = (cb & 0x7FFFFFu) >> mshift;
-        if (eh != ec) {
-            n_mis++;
-            n_large_m += (__usad(mh, mc, 0u) > static_cast<uint32_t>(p.e_m)) ? 1u : 0u;
-        } else {
-            // signed significands (implicit one unless the exponent field is zero), distance in steps
-            const uint32_t one = eh != 0u ? (1u << mbits) : 0u;
-            const uint32_t sh = one + mh, sc = one + mc;
-            const uint32_t dev = ((hb ^ cb) >> 31) ? sh + sc : __usad(sh, sc, 0u);
-            n_small_w += (static_cast<float>(dev) <= p.thr_w) ? 1u : 0u;
-            n_exact += (hb == cb) ? 1u : 0u;
-        }
+        n_small_w += (same_exp && dev <= p.thr_dev) ? 1u : 0u;
+        n_exact += (x == 0u) ? 1u : 0u;
+    }
+
+    // Two neighbouring elements against a packed pair of committed bf16 values (low half first).
+    __device__ __forceinline__ void add_bf16x2(float h_lo, float h_hi, uint32_t c_pair, const CmpParams& p) {
+        const uint32_t h_pair = pack_bf16(h_lo, h_hi);
+        add_bits(h_lo, h_pair << 16, c_pair << 16, p);
+        add_bits(h_hi, h_pair & 0xFFFF0000u, c_pair & 0xFFFF0000u, p);
+    }
+    __device__ __forceinline__ void add_f32(float h, uint32_t c_bits, const CmpParams& p) {
+        add_bits(h, __float_as_uint(h), c_bits, p);
     }
 
     __device__ __forceinline__ void store(float* dst) const {

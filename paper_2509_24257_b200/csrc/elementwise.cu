@@ -106,14 +106,10 @@ __global__ void compare_rows_kernel(const float* __restrict__ hidden, const void
             const uint4 cv = __ldg(c4 + j / 8);
             const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
             const float4 h1 = __ldg(reinterpret_cast<const float4*>(h + j + 4));
-            a.add<true>(h0.x, cv.x << 16, cmp);
-            a.add<true>(h0.y, cv.x & 0xFFFF0000u, cmp);
-            a.add<true>(h0.z, cv.y << 16, cmp);
-            a.add<true>(h0.w, cv.y & 0xFFFF0000u, cmp);
-            a.add<true>(h1.x, cv.z << 16, cmp);
-            a.add<true>(h1.y, cv.z & 0xFFFF0000u, cmp);
-            a.add<true>(h1.z, cv.w << 16, cmp);
-            a.add<true>(h1.w, cv.w & 0xFFFF0000u, cmp);
+            a.add_bf16x2(h0.x, h0.y, cv.x, cmp);
+            a.add_bf16x2(h0.z, h0.w, cv.y, cmp);
+            a.add_bf16x2(h1.x, h1.y, cv.z, cmp);
+            a.add_bf16x2(h1.z, h1.w, cv.w, cmp);
         }
     } else {
         const uint4* c4 =
@@ -121,10 +117,10 @@ __global__ void compare_rows_kernel(const float* __restrict__ hidden, const void
         for (int j = lane * 4; j < d; j += 128) {
             const uint4 cv = __ldg(c4 + j / 4);
             const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
-            a.add<false>(h0.x, cv.x, cmp);
-            a.add<false>(h0.y, cv.y, cmp);
-            a.add<false>(h0.z, cv.z, cmp);
-            a.add<false>(h0.w, cv.w, cmp);
+            a.add_f32(h0.x, cv.x, cmp);
+            a.add_f32(h0.y, cv.y, cmp);
+            a.add_f32(h0.z, cv.z, cmp);
+            a.add_f32(h0.w, cv.w, cmp);
         }
     }
     a.ss = warp_sum(a.ss);

@@ -202,6 +202,51 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t trow
     }
 }
 
+constexpr int EPI_STAGE_BYTES = 4 * 32 * 32 * 4;  // pair kernel: one 32 x 32 fp32 block per epilogue warp
+
+// Residual add of one tile with coalesced global traffic: each 32 x 32 block of the accumulator (one
+// row per lane) is transposed through a swizzled shared-memory block so that eight lanes cover the 128
+// contiguous bytes of one residual row.  `row0` is the first row of the warp's 32, `stage` its block.
+__device__ __forceinline__ void epilogue_resid_staged(const GemmParams& p, uint32_t trow, int row0, int n0, int lane,
+                                                      float4* stage) {
+    const int n_chunks = min(BN, p.N - n0) / 32;
+    const int sub = lane >> 3, c4 = lane & 7;
+    float* gbase = reinterpret_cast<float*>(p.out) + static_cast<size_t>(row0) * p.ldo + n0 + c4 * 4;
+    float4 nxt[8];
+    auto fetch = [&](int c, float4 (&dst)[8]) {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int r = it * 4 + sub;
+            if (row0 + r < p.M) dst[it] = *reinterpret_cast<const float4*>(gbase + static_cast<size_t>(r) * p.ldo + c * 32);
+        }
+    };
+    if (n_chunks > 0) fetch(0, nxt);
+#pragma unroll 1
+    for (int c = 0; c < n_chunks; ++c) {
+        float4 cur[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cur[i] = nxt[i];
+        if (c + 1 < n_chunks) fetch(c + 1, nxt);
+        float v[32];
+        load_acc(trow + c * 32, v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            stage[lane * 8 + (i ^ (lane & 7))] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        __syncwarp();
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int r = it * 4 + sub;
+            const float4 a = stage[r * 8 + (c4 ^ (r & 7))];
+            if (row0 + r < p.M) {
+                float4 x = cur[it];
+                x.x += a.x; x.y += a.y; x.z += a.z; x.w += a.w;
+                *reinterpret_cast<float4*>(gbase + static_cast<size_t>(r) * p.ldo + c * 32) = x;
+            }
+        }
+        __syncwarp();
+    }
+}
+
 // Gather-and-compare on the rows of this tile that carry check slots: the thread re-reads the 256
 // residual values it has just written, streams the committed values of each slot on the row
 // (16-byte loads) and leaves one partial record per (slot, column tile).
@@ -230,14 +275,10 @@ __device__ __forceinline__ void compare_row(const GemmParams& p, int row, int n0
                 const uint4 cv = __ldg(c4 + j / 8);
                 const float4 h0 = *reinterpret_cast<const float4*>(hrow + j);
                 const float4 h1 = *reinterpret_cast<const float4*>(hrow + j + 4);
-                acc.add<true>(h0.x, cv.x << 16, p.cmp);
-                acc.add<true>(h0.y, cv.x & 0xFFFF0000u, p.cmp);
-                acc.add<true>(h0.z, cv.y << 16, p.cmp);
-                acc.add<true>(h0.w, cv.y & 0xFFFF0000u, p.cmp);
-                acc.add<true>(h1.x, cv.z << 16, p.cmp);
-                acc.add<true>(h1.y, cv.z & 0xFFFF0000u, p.cmp);
-                acc.add<true>(h1.z, cv.w << 16, p.cmp);
-                acc.add<true>(h1.w, cv.w & 0xFFFF0000u, p.cmp);
+                acc.add_bf16x2(h0.x, h0.y, cv.x, p.cmp);
+                acc.add_bf16x2(h0.z, h0.w, cv.y, p.cmp);
+                acc.add_bf16x2(h1.x, h1.y, cv.z, p.cmp);
+                acc.add_bf16x2(h1.z, h1.w, cv.w, p.cmp);
                 if (hout) {
                     *reinterpret_cast<float4*>(hout + j) = h0;
                     *reinterpret_cast<float4*>(hout + j + 4) = h1;
@@ -250,10 +291,10 @@ __device__ __forceinline__ void compare_row(const GemmParams& p, int row, int n0
             for (int j = 0; j < ncols; j += 4) {
                 const uint4 cv = __ldg(c4 + j / 4);
                 const float4 h0 = *reinterpret_cast<const float4*>(hrow + j);
-                acc.add<false>(h0.x, cv.x, p.cmp);
-                acc.add<false>(h0.y, cv.y, p.cmp);
-                acc.add<false>(h0.z, cv.z, p.cmp);
-                acc.add<false>(h0.w, cv.w, p.cmp);
+                acc.add_f32(h0.x, cv.x, p.cmp);
+                acc.add_f32(h0.y, cv.y, p.cmp);
+                acc.add_f32(h0.z, cv.z, p.cmp);
+                acc.add_f32(h0.w, cv.w, p.cmp);
                 if (hout) *reinterpret_cast<float4*>(hout + j) = h0;
             }
         }
@@ -440,7 +481,7 @@ constexpr int P_STAGES = VL_PAIR_STAGES;
 constexpr int P_B_STAGE_BYTES = 128 * BK * 2;  // half of the B tile
 constexpr int P_STAGE_BYTES = A_STAGE_BYTES + P_B_STAGE_BYTES;
 constexpr int P_TILE_BYTES = P_STAGES * P_STAGE_BYTES;
-constexpr int P_GEMM_SMEM = P_TILE_BYTES + BAR_BYTES + 1024;
+constexpr int P_GEMM_SMEM = P_TILE_BYTES + BAR_BYTES + EPI_STAGE_BYTES + 1024;
 
 template <int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -580,7 +621,12 @@ gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             const int row = tc.m_idx * 2 * BM + static_cast<int>(rank) * BM + quarter * 32 + lane;
             const int n0 = tc.n_idx * BN;
             const uint32_t trow = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
-            epilogue_tile<EPI>(p, trow, row, n0, tc.n_idx);
+            if constexpr (EPI == EPI_RESID_ADD || EPI == EPI_RESID_ADD_COMPARE) {
+                float4* stage = reinterpret_cast<float4*>(smem_raw + (base - raw) + P_TILE_BYTES + BAR_BYTES) + quarter * 256;
+                epilogue_resid_staged(p, trow, row - lane, n0, lane, stage);
+            } else {
+                epilogue_tile<EPI>(p, trow, row, n0, tc.n_idx);
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(acc), 0));  // the leader collects all 8

@@ -152,12 +152,7 @@ TolDev tol_dev(const verillm_tol& t) {
 }
 
 CmpParams cmp_params(const verillm_tol& t, int commit_dtype) {
-    CmpParams c;
-    c.commit_dtype = commit_dtype;
-    c.tau_large = t.tau_large;
-    c.thr_w = t.e_w * static_cast<float>(1 << (commit_dtype == VERILLM_BF16 ? 7 : 23));
-    c.e_m = t.e_m;
-    return c;
+    return make_cmp_params(commit_dtype, t.tau_large, t.e_w, t.e_m);
 }
 
 // Checks the packed batch description; fills n_tokens and max_len.
