@@ -52,16 +52,22 @@ struct CmpAcc {
 
     // h: recomputed value (fp32); hb: h rounded to the commit dtype, as a float32 bit pattern; cb: the
     // committed value as a float32 bit pattern (a bf16 value widened by 16 zero bits, or the float32).
+    // kChecked = false leaves out the test for non-finite operands: the caller then inspects `sa` after
+    // the pass (any non-finite operand makes |h - c|, and with it the sum, non-finite) and repeats the
+    // pass with kChecked = true from cleared accumulators.
+    template <bool kChecked>
     __device__ __forceinline__ void add_bits(float h, uint32_t hb, uint32_t cb, const CmpParams& p) {
         const float c = __uint_as_float(cb);
         const float d = h - c;
         const float ad = fabsf(d);
-        if (!(ad < INFINITY)) {
-            // rare: a non-finite operand (counted and left out of every sum), or a finite pair whose
-            // difference overflowed (kept)
-            if ((__float_as_uint(h) & 0x7F800000u) == 0x7F800000u || (cb & 0x7F800000u) == 0x7F800000u) {
-                n_nonfinite++;
-                return;
+        if constexpr (kChecked) {
+            if (!(ad < INFINITY)) {
+                // a non-finite operand is counted and left out of every sum; a finite pair whose
+                // difference overflowed is kept
+                if ((__float_as_uint(h) & 0x7F800000u) == 0x7F800000u || (cb & 0x7F800000u) == 0x7F800000u) {
+                    n_nonfinite++;
+                    return;
+                }
             }
         }
         ss = fmaf(d, d, ss);
@@ -91,13 +97,15 @@ struct CmpAcc {
     }
 
     // Two neighbouring elements against a packed pair of committed bf16 values (low half first).
+    template <bool kChecked = true>
     __device__ __forceinline__ void add_bf16x2(float h_lo, float h_hi, uint32_t c_pair, const CmpParams& p) {
         const uint32_t h_pair = pack_bf16(h_lo, h_hi);
-        add_bits(h_lo, h_pair << 16, c_pair << 16, p);
-        add_bits(h_hi, h_pair & 0xFFFF0000u, c_pair & 0xFFFF0000u, p);
+        add_bits<kChecked>(h_lo, h_pair << 16, c_pair << 16, p);
+        add_bits<kChecked>(h_hi, h_pair & 0xFFFF0000u, c_pair & 0xFFFF0000u, p);
     }
+    template <bool kChecked = true>
     __device__ __forceinline__ void add_f32(float h, uint32_t c_bits, const CmpParams& p) {
-        add_bits(h, __float_as_uint(h), c_bits, p);
+        add_bits<kChecked>(h, __float_as_uint(h), c_bits, p);
     }
 
     __device__ __forceinline__ void store(float* dst) const {

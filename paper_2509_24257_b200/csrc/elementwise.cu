@@ -89,6 +89,34 @@ rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ ga
 }
 
 // ------------------------------------------------------------------ standalone comparison
+// One pass of a lane over its share of a row (16-byte loads, lanes interleaved).
+template <bool kChecked>
+__device__ __forceinline__ void compare_row_pass(CmpAcc& a, const float* __restrict__ h, const void* __restrict__ committed,
+                                                 size_t row, int d, int lane, const CmpParams& cmp) {
+    if (cmp.commit_dtype == VERILLM_BF16) {
+        const uint4* c4 = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(committed) + row * d);
+        for (int j = lane * 8; j < d; j += 256) {
+            const uint4 cv = __ldg(c4 + j / 8);
+            const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
+            const float4 h1 = __ldg(reinterpret_cast<const float4*>(h + j + 4));
+            a.add_bf16x2<kChecked>(h0.x, h0.y, cv.x, cmp);
+            a.add_bf16x2<kChecked>(h0.z, h0.w, cv.y, cmp);
+            a.add_bf16x2<kChecked>(h1.x, h1.y, cv.z, cmp);
+            a.add_bf16x2<kChecked>(h1.z, h1.w, cv.w, cmp);
+        }
+    } else {
+        const uint4* c4 = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(committed) + row * d);
+        for (int j = lane * 4; j < d; j += 128) {
+            const uint4 cv = __ldg(c4 + j / 4);
+            const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
+            a.add_f32<kChecked>(h0.x, cv.x, cmp);
+            a.add_f32<kChecked>(h0.y, cv.y, cmp);
+            a.add_f32<kChecked>(h0.z, cv.z, cmp);
+            a.add_f32<kChecked>(h0.w, cv.w, cmp);
+        }
+    }
+}
+
 // One warp per (layer, slot) row: coalesced 16-byte loads of both operands, per-lane accumulation,
 // fixed-order shuffle reduction, one partial record per row.
 __global__ void compare_rows_kernel(const float* __restrict__ hidden, const void* __restrict__ committed, int n_rows,
@@ -99,29 +127,12 @@ __global__ void compare_rows_kernel(const float* __restrict__ hidden, const void
     const float* h = hidden + static_cast<size_t>(row) * d;
     CmpAcc a;
     a.clear();
-    if (cmp.commit_dtype == VERILLM_BF16) {
-        const uint4* c4 = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(committed) +
-                                                         static_cast<size_t>(row) * d);
-        for (int j = lane * 8; j < d; j += 256) {
-            const uint4 cv = __ldg(c4 + j / 8);
-            const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
-            const float4 h1 = __ldg(reinterpret_cast<const float4*>(h + j + 4));
-            a.add_bf16x2(h0.x, h0.y, cv.x, cmp);
-            a.add_bf16x2(h0.z, h0.w, cv.y, cmp);
-            a.add_bf16x2(h1.x, h1.y, cv.z, cmp);
-            a.add_bf16x2(h1.z, h1.w, cv.w, cmp);
-        }
-    } else {
-        const uint4* c4 =
-            reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(committed) + static_cast<size_t>(row) * d);
-        for (int j = lane * 4; j < d; j += 128) {
-            const uint4 cv = __ldg(c4 + j / 4);
-            const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
-            a.add_f32(h0.x, cv.x, cmp);
-            a.add_f32(h0.y, cv.y, cmp);
-            a.add_f32(h0.z, cv.z, cmp);
-            a.add_f32(h0.w, cv.w, cmp);
-        }
+    // first pass without the per-element test for non-finite operands; any such operand leaves the sum
+    // of |h - c| non-finite, and the lane then repeats its share with the test
+    compare_row_pass<false>(a, h, committed, static_cast<size_t>(row), d, lane, cmp);
+    if (!(a.sa < INFINITY)) {
+        a.clear();
+        compare_row_pass<true>(a, h, committed, static_cast<size_t>(row), d, lane, cmp);
     }
     a.ss = warp_sum(a.ss);
     a.rr = warp_sum(a.rr);
@@ -204,7 +215,7 @@ __global__ void verdict_kernel(const float* __restrict__ partials, int n_layers,
 // One block per sequence, threads over check slots: accept iff all its checked positions were accepted (one
 // deviation above tolerance suffices to fail); score = mean MAE over its (slot, layer) cells.  Per-thread
 // double sums are combined by a fixed shuffle tree and then in warp order, so the result is reproducible.
-constexpr int kSeqThreads = 256;
+constexpr int kSeqThreads = 1024;
 __global__ void __launch_bounds__(kSeqThreads)
 seq_verdict_kernel(const float* __restrict__ stats, const uint8_t* __restrict__ pos_ok,
                    const int* __restrict__ seq_of_slot, int n_check, int n_layers, int batch,
