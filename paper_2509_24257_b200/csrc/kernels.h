@@ -58,7 +58,7 @@ cudaError_t gemm_init();  // raises the dynamic shared memory limit of every ins
 // tmap_q / tmap_kv are 64-column boxes of 128 / 64 rows over the same [tokens][(H+2KV)dh] buffer.
 cudaError_t launch_attention_tc(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, const int* cu_seqlens_dev,
                                 int batch, int max_seqlen, int n_heads, int n_kv_heads, int head_dim, void* out,
-                                int* status, cudaStream_t stream);
+                                int* status, int num_sms, cudaStream_t stream);
 cudaError_t attention_tc_init();
 
 // ------------------------------------------------------------------ small kernels

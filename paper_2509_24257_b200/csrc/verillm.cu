@@ -222,7 +222,7 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
     CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, p.pair ? w.t_wqkv_h : w.t_wqkv, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_QKV, st);
     CU_TRY(launch_attention_tc(m->t_qkv_q, m->t_qkv_kv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads,
-                               c.head_dim, m->attn, status, st));
+                               c.head_dim, m->attn, status, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_ATTENTION, st);
     p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
     p.group_m = band_d;
@@ -913,8 +913,11 @@ int verillm_op_attention(const void* qkv, const int32_t* cu_seqlens, int32_t bat
     CUtensorMap tq, tkv;
     if (make_tmap_bf16_2d(&tq, qkv, M, n_qkv, n_qkv, 128) != 0) return VERILLM_E_CUDA;
     if (make_tmap_bf16_2d(&tkv, qkv, M, n_qkv, n_qkv, 64) != 0) return VERILLM_E_CUDA;
+    int dev = 0, num_sms = 0;
+    CU_TRY(cudaGetDevice(&dev));
+    CU_TRY(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
     CU_TRY(launch_attention_tc(tq, tkv, cu_seqlens, batch, max_seqlen, n_heads, n_kv_heads, head_dim, out, nullptr,
-                               reinterpret_cast<cudaStream_t>(cuda_stream)));
+                               num_sms, reinterpret_cast<cudaStream_t>(cuda_stream)));
     return VERILLM_OK;
 }
 
