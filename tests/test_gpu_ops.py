@@ -68,6 +68,31 @@ def test_attention_matches_oracle(Hq, KV, dh, lens):
         assert np.array_equal(got[0], v[0, [g * KV // Hq for g in range(Hq)]])  # first row = v_0 exactly
 
 
+def test_attention_many_units_per_cta():
+    """More (sequence, head, query tile) units than the persistent CTAs keep in their shared-memory table, so the
+    later units are looked up on the spot, over several dealing rounds: sampled sequences against the oracle,
+    and the closed form row 0 = v_0 on every sequence and head."""
+    Hq, KV, dh = 32, 8, 64
+    rng = np.random.default_rng(77)
+    lens = rng.integers(1, 161, size=480)
+    lens[:4] = [160, 129, 128, 1]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    assert 2 * Hq * len(lens) > 48 * 2 * torch.cuda.get_device_properties(0).multi_processor_count
+    qkv = _rand_bf16((int(cu[-1]), (Hq + 2 * KV) * dh), 12, 1.0)
+    out = vb.op_attention(qkv.to(DEV), cu, Hq, KV, dh).float().cpu().numpy().astype(np.float64)
+    x = vo.as_f64(H.bits(qkv))
+    assert np.all(np.isfinite(out))
+    v_first = x[cu[:-1], (Hq + KV) * dh :].reshape(len(lens), KV, dh)
+    assert np.array_equal(out[cu[:-1]].reshape(len(lens), Hq, dh), v_first[:, [g * KV // Hq for g in range(Hq)]])
+    for b in list(range(4)) + rng.choice(len(lens), 12, replace=False).tolist():
+        s, e = int(cu[b]), int(cu[b + 1])
+        q = x[s:e, : Hq * dh].reshape(-1, Hq, dh)
+        k = x[s:e, Hq * dh : (Hq + KV) * dh].reshape(-1, KV, dh)
+        v = x[s:e, (Hq + KV) * dh :].reshape(-1, KV, dh)
+        ref = vo.causal_attention(q, k, v).reshape(e - s, Hq, dh)
+        assert np.max(H.rel_l2(out[s:e].reshape(e - s, Hq, dh), ref)) <= 1e-2
+
+
 def _engineered_pairs(d, seed):
     """Hidden/committed rows that exercise every branch of the comparison."""
     rng = np.random.default_rng(seed)
