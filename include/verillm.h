@@ -237,6 +237,19 @@ int verillm_spot_check(const float *hidden, int32_t n_rows, int32_t d_model, con
                        const int32_t *sample_col, const float *reference, int32_t n_samples, float eps, float theta,
                        uint8_t *agree_out, float *p_hat_out, uint8_t *verdict_out, void *cuda_stream);
 
+/* Threshold sensitivity of the offline tests ("Threshold Sensitivity Analysis": each threshold is varied while the
+ * others stay at their selected values, and the false-positive / false-negative rates are read off honest and
+ * attack traces).  The tests of the verdict are applied to statistics reported by an earlier verify / compare call.
+ *  stats      DEVICE float32 [n_cells][VERILLM_NSTAT]: one row per (position, layer) cell, as written to report.stats
+ *  is_attack  DEVICE uint8 [n_cells]: 0 = the cell comes from an honest trace, non-zero = from an attack trace
+ *  variants   HOST verillm_tol [n_variants], 1 <= n_variants <= 64 (E_SHAPE beyond): the tolerance sets to evaluate;
+ *             tau_large, e_w and e_m are not used (they shaped the statistics when these were produced)
+ *  counts_out DEVICE int32 [n_variants][4], zeroed by the call: honest accepted, honest rejected, attack accepted,
+ *             attack rejected.  FPR = honest rejected / honest, FNR = attack accepted / attack.
+ * A cell with a non-finite element is rejected by every variant.  Allocates nothing. */
+int verillm_threshold_sweep(const float *stats, const uint8_t *is_attack, int32_t n_cells, const verillm_tol *variants,
+                            int32_t n_variants, int32_t *counts_out, void *cuda_stream);
+
 /* Merkle commitment of hidden states ("serializes its output tensor, constructs a Merkle tree over all scalar
  * entries and submits the Merkle root"; canonical float32 leaves, SHA-256): one root per vector.
  *  states    DEVICE float32 [n_vec][d_model]; roots_out DEVICE uint8 [n_vec][32]

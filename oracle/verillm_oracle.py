@@ -381,6 +381,32 @@ def layer_passes(stats: np.ndarray, tol: Tol) -> np.ndarray:
     return ok
 
 
+def threshold_sweep(stats: np.ndarray, is_attack: np.ndarray, variants: Sequence[Tol]) -> np.ndarray:
+    """Threshold Sensitivity Analysis: for each tolerance set, how many honest and attack cells its tests accept
+    and reject.  stats: [n_cells, NSTAT]; is_attack: [n_cells] bool.  Returns int64 [n_variants, 4] = honest
+    accepted, honest rejected, attack accepted, attack rejected.  The thresholds are taken at float32
+    precision, the precision a GPU verifier holds them in (the statistics it reports are float32 too)."""
+    stats = np.asarray(stats, dtype=np.float64).reshape(-1, NSTAT)
+    attack = np.asarray(is_attack).astype(bool).reshape(-1)
+    out = np.zeros((len(variants), 4), dtype=np.int64)
+    for v, tol in enumerate(variants):
+        t32 = dataclasses.replace(tol, **{f.name: float(np.float32(getattr(tol, f.name)))
+                                          for f in dataclasses.fields(tol) if isinstance(getattr(tol, f.name), float)})
+        ok = layer_passes(stats, t32)
+        out[v] = [np.sum(ok & ~attack), np.sum(~ok & ~attack), np.sum(ok & attack), np.sum(~ok & attack)]
+    return out
+
+
+def detection_rates(counts: np.ndarray) -> Dict[str, np.ndarray]:
+    """FPR / FNR / TPR / TNR of the table in Threshold Sensitivity Analysis from threshold_sweep's counts
+    (positive = attack detected, i.e. rejected)."""
+    c = np.asarray(counts, dtype=np.float64)
+    honest, attack = c[:, 0] + c[:, 1], c[:, 2] + c[:, 3]
+    with np.errstate(invalid="ignore", divide="ignore"):
+        fpr, fnr = c[:, 1] / honest, c[:, 2] / attack
+    return {"FPR": fpr, "FNR": fnr, "TPR": 1.0 - fnr, "TNR": 1.0 - fpr}
+
+
 @dataclasses.dataclass
 class Report:
     stats: np.ndarray  # [n_check, n_layers, NSTAT]

@@ -31,6 +31,7 @@ EXPORTS = (
     "verillm_op_rmsnorm", "verillm_op_attention", "verillm_free", "verillm_strerror",
     "verillm_last_launch_count", "verillm_profile_enable", "verillm_profile_read",
     "verillm_load_lm_head", "verillm_token_match", "verillm_verify_segment", "verillm_spot_check", "verillm_merkle_roots",
+    "verillm_threshold_sweep",
 )
 PROF_CLASSES = ("setup", "rmsnorm", "gemm_qkv_rope", "attention", "gemm_o_resid", "gemm_gate_up_swiglu",
                 "gemm_down_resid_compare", "verdict")
@@ -119,6 +120,8 @@ def lib() -> C.CDLL:
         L.verillm_spot_check.restype = C.c_int
         L.verillm_merkle_roots.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.verillm_merkle_roots.restype = C.c_int
+        L.verillm_threshold_sweep.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(Tol), C.c_int32, C.c_void_p, C.c_void_p]
+        L.verillm_threshold_sweep.restype = C.c_int
         L.verillm_load_lm_head.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
         L.verillm_load_lm_head.restype = C.c_int
         L.verillm_token_match.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -407,6 +410,22 @@ def spot_check(hidden: torch.Tensor, sample_row, sample_col, reference, eps: flo
                                         cols.ctypes.data, ref.ctypes.data, n, float(eps), float(theta), agree.data_ptr(),
                                         p_hat.data_ptr(), ok.data_ptr(), _stream_ptr(stream)), "verillm_spot_check")
     return agree, p_hat, ok
+
+
+def threshold_sweep(stats: torch.Tensor, is_attack: torch.Tensor, variants: Sequence[Tol],
+                    stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """stats float32 device [n_cells][NSTAT] (report.stats reshaped), is_attack uint8 device [n_cells], up to 64
+    tolerance sets -> int32 device [n_variants][4] = honest accepted, honest rejected, attack accepted, attack rejected."""
+    if stats.dtype != torch.float32 or not stats.is_contiguous() or stats.dim() != 2 or stats.shape[1] != NSTAT:
+        raise ValueError("stats must be a contiguous float32 [n_cells][NSTAT] tensor")
+    if is_attack.dtype != torch.uint8 or not is_attack.is_contiguous() or is_attack.numel() != stats.shape[0]:
+        raise ValueError("is_attack must be a contiguous uint8 tensor with one entry per cell")
+    arr = (Tol * len(variants))(*variants)
+    counts = torch.empty(len(variants), 4, dtype=torch.int32, device=stats.device)
+    with torch.cuda.device(stats.device):
+        _check(lib().verillm_threshold_sweep(stats.data_ptr(), is_attack.data_ptr(), stats.shape[0], arr, len(variants),
+                                             counts.data_ptr(), _stream_ptr(stream)), "verillm_threshold_sweep")
+    return counts
 
 
 def merkle_roots(states: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:

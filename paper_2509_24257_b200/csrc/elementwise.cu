@@ -212,6 +212,55 @@ __global__ void verdict_kernel(const float* __restrict__ partials, int n_layers,
     }
 }
 
+// ------------------------------------------------------------------ threshold sensitivity
+// The tests of verdict_kernel applied to statistics that were reported earlier: one thread per (position,
+// layer) cell reads its VERILLM_NSTAT floats once and evaluates every tolerance variant; per variant the block
+// counts accepted / rejected cells of the honest and of the attack class (warp ballots, integer atomics).
+__device__ __forceinline__ bool stats_pass(const float4& s0, const float4& s1, const float4& s2, const float4& s3,
+                                           const TolDev& tol) {
+    bool ok = s3.y == 0.f;  // no non-finite element
+    if (tol.rel_l2 > 0.f) ok = ok && (s0.x <= tol.rel_l2);
+    if (tol.max_abs > 0.f) ok = ok && (s0.y <= tol.max_abs);
+    if (tol.mae > 0.f) ok = ok && (s0.z <= tol.mae);
+    if (tol.z_large_max >= 0.f) ok = ok && (s2.x <= tol.z_large_max);
+    if (tol.q_small_min > 0.f) ok = ok && (s1.w >= tol.q_small_min);
+    if (tol.bit_aware)
+        ok = ok && (s1.x < tol.pe_max) && (s1.y > tol.pm_min) && (s1.z > tol.pw_min) && (fabsf(s0.w) <= tol.e_abs_max);
+    return ok;
+}
+
+__global__ void __launch_bounds__(256)
+threshold_sweep_kernel(const float* __restrict__ stats, const uint8_t* __restrict__ is_attack, int n_cells,
+                       const __grid_constant__ TolSet tols, int n_variants, int* __restrict__ counts) {
+    const int cell = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool live = cell < n_cells;
+    float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0, s2 = s0, s3 = s0;
+    bool attack = false;
+    if (live) {
+        const float4* p = reinterpret_cast<const float4*>(stats + static_cast<size_t>(cell) * VERILLM_NSTAT);
+        s0 = __ldg(p);
+        s1 = __ldg(p + 1);
+        s2 = __ldg(p + 2);
+        s3 = __ldg(p + 3);
+        attack = is_attack[cell] != 0;
+    }
+    const int lane = threadIdx.x & 31;
+#pragma unroll 1
+    for (int v = 0; v < n_variants; ++v) {
+        const bool ok = stats_pass(s0, s1, s2, s3, tols.v[v]);
+        const uint32_t ha = __ballot_sync(0xFFFFFFFFu, live && !attack && ok);
+        const uint32_t hr = __ballot_sync(0xFFFFFFFFu, live && !attack && !ok);
+        const uint32_t aa = __ballot_sync(0xFFFFFFFFu, live && attack && ok);
+        const uint32_t ar = __ballot_sync(0xFFFFFFFFu, live && attack && !ok);
+        if (lane == 0) {
+            if (ha) atomicAdd(counts + 4 * v + 0, __popc(ha));
+            if (hr) atomicAdd(counts + 4 * v + 1, __popc(hr));
+            if (aa) atomicAdd(counts + 4 * v + 2, __popc(aa));
+            if (ar) atomicAdd(counts + 4 * v + 3, __popc(ar));
+        }
+    }
+}
+
 // One block per sequence, threads over check slots: accept iff all its checked positions were accepted (one
 // deviation above tolerance suffices to fail); score = mean MAE over its (slot, layer) cells.  Per-thread
 // double sums are combined by a fixed shuffle tree and then in warp order, so the result is reproducible.
@@ -569,6 +618,13 @@ cudaError_t launch_seq_verdict(const float* stats, const uint8_t* pos_ok, const 
     if (batch <= 0) return cudaSuccess;
     seq_verdict_kernel<<<batch, kSeqThreads, 0, s>>>(stats, pos_ok, seq_of_slot, n_check, n_layers, batch, seq_ok,
                                                         seq_score);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_threshold_sweep(const float* stats, const uint8_t* is_attack, int n_cells, const TolSet& tols,
+                                   int n_variants, int* counts, cudaStream_t s) {
+    if (n_cells <= 0 || n_variants <= 0) return cudaSuccess;
+    threshold_sweep_kernel<<<(n_cells + 255) / 256, 256, 0, s>>>(stats, is_attack, n_cells, tols, n_variants, counts);
     return cudaGetLastError();
 }
 

@@ -85,6 +85,15 @@ cudaError_t launch_verdict(const float* partials, int n_layers, int n_check, int
 cudaError_t launch_seq_verdict(const float* stats, const uint8_t* pos_ok, const int* seq_of_slot, int n_check,
                                int n_layers, int batch, uint8_t* seq_ok, float* seq_score, cudaStream_t stream);
 
+// Threshold sensitivity: counts[v][4] += (honest accepted, honest rejected, attack accepted, attack rejected)
+// over the cells' reported statistics [n_cells][VERILLM_NSTAT] for each of n_variants tolerance sets.
+constexpr int kSweepMaxVariants = 64;
+struct TolSet {
+    TolDev v[kSweepMaxVariants];
+};
+cudaError_t launch_threshold_sweep(const float* stats, const uint8_t* is_attack, int n_cells, const TolSet& tols,
+                                   int n_variants, int* counts, cudaStream_t stream);
+
 // Tail token check: reduces the per-tile argmax records of the output-head product [rows][n_tiles][4] (fixed order,
 // lowest column wins ties), compares with the claimed tokens.
 cudaError_t launch_argmax_reduce(const float* records, int rows, int n_tiles, const int* claimed, int* argmax_out,

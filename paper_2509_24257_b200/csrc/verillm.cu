@@ -714,6 +714,19 @@ int verillm_spot_check(const float* hidden, int32_t n_rows, int32_t d_model, con
     return VERILLM_OK;
 }
 
+int verillm_threshold_sweep(const float* stats, const uint8_t* is_attack, int32_t n_cells, const verillm_tol* variants,
+                            int32_t n_variants, int32_t* counts_out, void* cuda_stream) {
+    if (!stats || !is_attack || !variants || !counts_out || n_cells < 1 || n_variants < 1) return VERILLM_E_INVAL;
+    if (n_variants > kSweepMaxVariants) return VERILLM_E_SHAPE;
+    TolSet set;
+    std::memset(&set, 0, sizeof(set));
+    for (int v = 0; v < n_variants; ++v) set.v[v] = tol_dev(variants[v]);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    CU_TRY(cudaMemsetAsync(counts_out, 0, sizeof(int32_t) * 4 * n_variants, st));
+    CU_TRY(launch_threshold_sweep(stats, is_attack, n_cells, set, n_variants, counts_out, st));
+    return VERILLM_OK;
+}
+
 int verillm_merkle_roots(const float* states, int32_t n_vec, int32_t d_model, uint8_t* roots_out, void* cuda_stream) {
     if (!states || !roots_out || n_vec < 1 || d_model < 1) return VERILLM_E_INVAL;
     if (d_model > 12800) return VERILLM_E_SHAPE;  // one level of the tree must fit in shared memory

@@ -295,6 +295,22 @@ def model_weights(
     }
 
 
+def fake_quantise(w: torch.Tensor, bits: int = 8) -> torch.Tensor:
+    """Weights of a prover that serves a quantised model (the quantisation attack): every output row is
+    rounded to a symmetric `bits`-bit integer grid spanning its largest magnitude, and widened back to the
+    tensor's dtype.  Input recipe of the attack traces only; the verifier never sees these weights."""
+    w32 = w.to(torch.float32)
+    qmax = float(2 ** (bits - 1) - 1)
+    scale = w32.abs().amax(dim=-1, keepdim=True).clamp_min(1e-30) / qmax
+    return (torch.round(w32 / scale).clamp_(-qmax, qmax) * scale).to(w.dtype)
+
+
+def quantised_model_weights(weights: Dict[str, object], bits: int = 8) -> Dict[str, object]:
+    """The same model with every projection matrix fake-quantised (norm gains and the embedding untouched)."""
+    layers = [{k: (v if k.endswith("norm") else fake_quantise(v, bits)) for k, v in lw.items()} for lw in weights["layers"]]
+    return {"embed": weights["embed"], "final_norm": weights["final_norm"], "layers": layers}
+
+
 # --------------------------------------------------------------------------- sequences
 
 

@@ -486,3 +486,76 @@ def test_merkle_root_structure_and_inclusion_proofs():
     two = vo.merkle_root(np.array([1.0, 2.0]))
     assert two == hashlib.sha256(hashlib.sha256(bytes.fromhex("0000803f")).digest()
                                  + hashlib.sha256(bytes.fromhex("00000040")).digest()).digest()
+
+
+# ----------------------------------------------------------------------------- threshold sensitivity
+
+
+def _cell(**kw):
+    row = np.zeros(vo.NSTAT)
+    row[vo.STAT_NAMES.index("p_m")] = 1.0
+    row[vo.STAT_NAMES.index("p_w")] = 1.0
+    for k, v in kw.items():
+        row[vo.STAT_NAMES.index(k)] = v
+    return row
+
+
+def test_threshold_sweep_hand_worked_cells():
+    """Seven cells whose verdict under three tolerance sets is worked out by hand (strict P_e / P_m / P_w,
+    closed |e| and rel-L2 intervals, a non-finite element rejects, equality with a strict bound rejects)."""
+    f32 = lambda x: float(np.float32(x))
+    stats = np.stack([
+        _cell(rel_l2=0.01, p_e=0.01, p_m=1.0, p_w=0.9, mean_signed=0.001),     # honest, clean
+        _cell(rel_l2=0.03, p_e=0.06, p_m=0.8, p_w=0.85),                       # honest, P_e above 0.05
+        _cell(rel_l2=0.01, p_e=0.02, p_m=0.7, p_w=0.95, mean_signed=-0.02),    # honest, P_m low and |e| high
+        _cell(rel_l2=0.0, p_e=f32(0.05)),                                      # honest, P_e exactly at the strict bound
+        _cell(rel_l2=0.02, p_e=0.08, p_m=0.95, p_w=0.3),                       # attack inside the rel-L2 tolerance
+        _cell(rel_l2=0.2, p_e=0.5, p_m=0.9, p_w=0.05),                         # gross attack
+        _cell(rel_l2=0.01, p_e=0.01, p_m=1.0, p_w=0.9, n_nonfinite=1),         # attack hiding behind a NaN
+    ])
+    attack = np.array([0, 0, 0, 0, 1, 1, 1], dtype=bool)
+    variants = [
+        vo.Tol(),                                                                               # rel-L2 <= 5e-2 only
+        vo.Tol(bit_aware=True),                                                                 # + the paper's selected set
+        vo.Tol(rel_l2=0.0, bit_aware=True, pe_max=0.07, pm_min=0.6, pw_min=0.5, e_abs_max=0.05),
+    ]
+    counts = vo.threshold_sweep(stats, attack, variants)
+    assert counts.tolist() == [[4, 0, 1, 2], [1, 3, 0, 3], [4, 0, 0, 3]]
+    r = vo.detection_rates(counts)
+    assert r["FPR"].tolist() == [0.0, 0.75, 0.0] and r["FNR"].tolist() == [1 / 3, 0.0, 0.0]
+    assert np.allclose(r["TPR"] + r["FNR"], 1.0) and np.allclose(r["TNR"] + r["FPR"], 1.0)
+
+
+def test_threshold_sweep_is_monotone_and_agrees_with_the_verdict():
+    rng = np.random.default_rng(5)
+    n = 400
+    stats = np.zeros((n, vo.NSTAT))
+    for name, lo, hi in (("rel_l2", 0, 0.1), ("p_e", 0, 0.2), ("p_m", 0.4, 1), ("p_w", 0, 1), ("mean_signed", -0.03, 0.03)):
+        stats[:, vo.STAT_NAMES.index(name)] = rng.uniform(lo, hi, n).astype(np.float32)
+    attack = rng.random(n) < 0.5
+    base = dict(rel_l2=0.0, bit_aware=True)
+    # loosening a threshold never turns an accept into a reject
+    for field, values in (("pe_max", (0.02, 0.05, 0.1)), ("pm_min", (0.9, 0.75, 0.5)), ("pw_min", (0.9, 0.8, 0.3)),
+                          ("e_abs_max", (0.005, 0.01, 0.02))):
+        c = vo.threshold_sweep(stats, attack, [vo.Tol(**base, **{field: v}) for v in values])
+        assert np.all(np.diff(c[:, 0]) >= 0) and np.all(np.diff(c[:, 2]) >= 0)
+        assert np.all(c.sum(axis=1) == n)
+    # one layer per position: a cell passes the sweep iff the position verdict accepts it
+    tol = vo.Tol(bit_aware=True)
+    pos_ok, _, _, _ = vo.verdict(stats.reshape(n, 1, vo.NSTAT), np.zeros(n, dtype=np.int32), 1, tol)
+    c = vo.threshold_sweep(stats, np.zeros(n, dtype=bool), [tol])
+    assert c[0, 0] == int(pos_ok.sum()) and c[0, 1] == n - int(pos_ok.sum())
+
+
+def test_fake_quantise_grid_and_error_bound():
+    """The attack model of the sensitivity analysis: values land on a symmetric integer grid per row, the row
+    maximum is kept, and the error is at most half a step."""
+    w = torch.from_numpy(np.random.default_rng(3).standard_normal((7, 64)).astype(np.float32))
+    for bits in (8, 4):
+        q = synth.fake_quantise(w, bits)
+        qmax = 2 ** (bits - 1) - 1
+        step = w.abs().amax(dim=1, keepdim=True) / qmax
+        k = q / step
+        assert torch.allclose(k, torch.round(k), atol=1e-4) and float(k.abs().max()) <= qmax + 1e-4
+        assert float(((q - w).abs() / step).max()) <= 0.5 + 1e-5
+        assert torch.allclose(q.abs().amax(dim=1), w.abs().amax(dim=1))
