@@ -2,12 +2,13 @@
 // in tensor memory, and the fused epilogues of the verifier's layer (rotary embedding, residual add,
 // SwiGLU, gather-and-compare).  These are the projections inside F_i of S_{i+1} = F_i(S_i; W_i).
 //
-// One persistent CTA per SM walks a list of 128 x 256 output tiles.  Warp 0 feeds a 4-stage ring of
-// shared-memory tiles with TMA (128-byte swizzle), warp 1 issues tcgen05.mma (one thread) into one of
-// two 256-column TMEM accumulators, warps 2-5 drain the other accumulator (tcgen05.ld, one output row
-// per thread) and run the epilogue, so the epilogue of a tile overlaps the main loop of the next.
-// Every mbarrier wait is bounded; a wait that runs out records VERILLM_DEV_WAIT_TIMEOUT and the CTA
-// falls through to its tail, which frees the tensor memory.
+// Two kernels share the epilogues.  For M > 128 rows, clusters of two CTAs on neighbouring SMs share one
+// 256 x 256 output tile (tcgen05.mma.cta_group::2; see gemm_bf16_tcgen05_pair below); for M <= 128 one
+// persistent CTA per SM walks 128 x 256 tiles.  In both, warp 0 feeds a ring of shared-memory tiles with TMA
+// (128-byte swizzle), warp 1 issues tcgen05.mma (one thread) into one of two 256-column TMEM accumulators,
+// warps 2-5 drain the other accumulator (tcgen05.ld, one output row per thread) and run the epilogue, so the
+// epilogue of a tile overlaps the main loop of the next.  Every mbarrier wait is bounded; a wait that runs out
+// records VERILLM_DEV_WAIT_TIMEOUT and the CTA falls through to its tail, which frees the tensor memory.
 #include "kernels.h"
 
 namespace vl {
@@ -474,10 +475,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 // by a third and leaves room for a 6-stage ring.  Barrier protocol: both CTAs' TMA loads count on the
 // leader's full barrier; the leader's tcgen05.commit releases the stage / publishes the accumulator in
 // both CTAs; the epilogue warps of both CTAs report the accumulator drained on the leader's barrier.
-#ifndef VL_PAIR_STAGES
-#define VL_PAIR_STAGES 6
-#endif
-constexpr int P_STAGES = VL_PAIR_STAGES;
+constexpr int P_STAGES = 6;
 constexpr int P_B_STAGE_BYTES = 128 * BK * 2;  // half of the B tile
 constexpr int P_STAGE_BYTES = A_STAGE_BYTES + P_B_STAGE_BYTES;
 constexpr int P_TILE_BYTES = P_STAGES * P_STAGE_BYTES;
