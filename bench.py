@@ -30,6 +30,7 @@ sys.path.insert(0, ROOT)
 METRIC, UNIT = "verified_tokens_per_sec", "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 TOL_REL_L2 = 5e-2
+SHA256_INT_OPS = 64 * 14 + 48 * 10 + 8  # 32-bit integer instructions of one compression
 GATE_UP_DRAM_BYTES_8B = 648.9e6 + 226.4e6  # measured, per launch, M = 8192 tokens at the 8B widths
 
 
@@ -411,9 +412,17 @@ def run_ours(args, wl):
     torch.cuda.synchronize()
     mk_ms = m0.elapsed_time(m1) / 5
     n_compress = mk_in.shape[0] * (4 * ((s.d_model + 1) // 2) + 2 * ((s.d_model + 1) // 2 - 1))
+    # ALU peak: one SHA-256 compression is 1384 32-bit integer instructions as written (64 rounds x 14, 48 schedule
+    # words x 10, 8 final adds); an SM issues 4 warp instructions = 128 lane operations per clock
+    props = torch.cuda.get_device_properties(device)
+    sm_clock_hz = 1e6 * float(clocks.get("sm_max_mhz") or 1965.0)
+    mk_peak = props.multi_processor_count * 128 * sm_clock_hz / SHA256_INT_OPS
+    mk_rate = n_compress / (mk_ms * 1e-3)
     merkle = {"vectors": int(mk_in.shape[0]), "scalars_per_vector": s.d_model, "ms": round(mk_ms, 4), "bound": "alu",
               "ns_per_scalar": round(mk_ms * 1e6 / mk_in.numel(), 4),
-              "sha256_compressions_per_s": round(n_compress / (mk_ms * 1e-3), 0)}
+              "sha256_compressions_per_s": round(mk_rate, 0), "peak_compressions_per_s": round(mk_peak, 0),
+              "frac": round(mk_rate / mk_peak, 4),
+              "peak_kind": "derived: SMs x 128 integer lane-ops per clock x max SM clock / 1384 ops per compression"}
     del mk_in
 
     if rank == 0:
