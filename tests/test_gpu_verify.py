@@ -198,6 +198,26 @@ def test_small_honest_trace(small):
     assert g["pos_ok"].all() and g["seq_ok"].all()
 
 
+def test_small_ragged_batch_spanning_several_row_tiles(small):
+    """890 packed tokens = three full 256-row tiles and a ragged one through the CTA-pair GEMMs (coalesced
+    residual epilogue, fused compare), sequences that end inside a tile, checks on first and last rows."""
+    wl, _, om, _, _, _, model, _, _ = small
+    rng = np.random.default_rng(17)
+    lens = [300, 77, 513]
+    seqs = [rng.integers(0, wl.shape.vocab, n).astype(np.int32) for n in lens]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    cs = np.array([2, 0, 1, 2, 0, 2], dtype=np.int32)
+    cp = np.array([512, 299, 76, 0, 0, 255], dtype=np.int32)
+    committed = np.zeros((wl.shape.n_layers, len(cs), wl.shape.d_model))
+    for i, (b, q) in enumerate(zip(cs, cp)):
+        committed[:, i] = vo.forward_decode_kvcache(om, seqs[b][: q + 1], "bf16")[:, q]
+    committed = synth.add_state_noise(committed, [0], [wl.shape.n_layers - 1], 10 * TOL, rng)
+    g, o = run_both(model, om, wl, None, committed, cs, cp, seqs=seqs, cu=cu)
+    assert_parity(g, o, expect_reject=[0])
+    assert g["pos_ok"].tolist() == [0, 1, 1, 1, 1, 1] and g["first_bad_layer"][0] == wl.shape.n_layers - 1
+    assert g["seq_ok"].tolist() == [1, 1, 0]
+
+
 def test_small_substituted_token_is_caught_at_its_position(small):
     wl, tokens, om, cs, cp, committed, model, rng, (sq, sp) = small
     forged = synth.swap_token(tokens, sq, sp, wl.shape.vocab, rng)
