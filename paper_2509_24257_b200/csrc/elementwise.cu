@@ -88,6 +88,36 @@ rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ ga
     }
 }
 
+// Unnormalised half of a folded norm: y = bf16(x * gain) and the row's sum of squares (see GemmParams).
+__global__ void __launch_bounds__(kNormThreads)
+prenorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ y,
+               float* __restrict__ sumsq, int n_parts, int d) {
+    const int row = blockIdx.x;
+    const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(row) * d);
+    uint2* yr = reinterpret_cast<uint2*>(y + static_cast<size_t>(row) * d);
+    const uint2* g2 = reinterpret_cast<const uint2*>(gain);
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d / 4; i += kNormThreads) {
+        const float4 v = xr[i];
+        const uint2 g = __ldg(g2 + i);
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        uint2 o;
+        o.x = pack_bf16(v.x * bf16_lo(g.x), v.y * bf16_hi(g.x));
+        o.y = pack_bf16(v.z * bf16_lo(g.y), v.w * bf16_hi(g.y));
+        yr[i] = o;
+    }
+    __shared__ float warp_part[kNormThreads / 32];
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < kNormThreads / 32; ++w) t += warp_part[w];
+        sumsq[static_cast<size_t>(row) * n_parts] = t;
+    }
+    for (int k = 1 + threadIdx.x; k < n_parts; k += kNormThreads) sumsq[static_cast<size_t>(row) * n_parts + k] = 0.f;
+}
+
 // ------------------------------------------------------------------ standalone comparison
 // One pass of a lane over its share of a row (16-byte loads, lanes interleaved).
 template <bool kChecked>
@@ -595,6 +625,14 @@ cudaError_t launch_rmsnorm(const float* x, const void* gain, void* y, int rows, 
     if (rows <= 0) return cudaSuccess;
     rmsnorm_kernel<<<rows, kNormThreads, 0, s>>>(x, reinterpret_cast<const __nv_bfloat16*>(gain),
                                                  reinterpret_cast<__nv_bfloat16*>(y), d, eps);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prenorm(const float* x, const void* gain, void* y, float* sumsq, int n_parts, int rows, int d,
+                           cudaStream_t s) {
+    if (rows <= 0) return cudaSuccess;
+    prenorm_kernel<<<rows, kNormThreads, 0, s>>>(x, reinterpret_cast<const __nv_bfloat16*>(gain),
+                                                 reinterpret_cast<__nv_bfloat16*>(y), sumsq, n_parts, d);
     return cudaGetLastError();
 }
 

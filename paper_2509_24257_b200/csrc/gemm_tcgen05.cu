@@ -69,6 +69,16 @@ __device__ __forceinline__ void load_acc(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Factor of a folded RMSNorm for one row: rsqrt(mean x^2 + eps) from the producer's per-tile sums of squares,
+// added in index order (1 when the projection's input was normalised beforehand).
+__device__ __forceinline__ float row_rstd(const GemmParams& p, int row, bool row_ok) {
+    if (p.sumsq_in == nullptr || !row_ok) return 1.f;
+    const float* s = p.sumsq_in + static_cast<size_t>(row) * p.n_parts;
+    float t = 0.f;
+    for (int k = 0; k < p.n_parts; ++k) t += s[k];
+    return rsqrtf(t * p.norm_inv_d + p.norm_eps);
+}
+
 // Epilogue of one tile for one thread (= one output row).  `trow` is the TMEM address of the thread's
 // lane at column 0 of the accumulator.  tcgen05.ld is warp-collective: every branch that contains one
 // is uniform across the warp (it depends on the tile only); row validity only predicates memory traffic.
@@ -158,6 +168,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t trow
         const int dh = p.head_dim;
         const int half_chunks = dh / 64;  // 32-column chunks per half head: 1 (dh 64) or 2 (dh 128)
         const int pos = row_ok ? p.pos_of_token[row] : 0;
+        const float rs = row_rstd(p, row, row_ok);
         __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<size_t>(row_ok ? row : 0) * p.ldo;
 #pragma unroll 1
         for (int hb = 0; hb < BN; hb += dh) {
@@ -175,9 +186,15 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t trow
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const float2 t = __ldg(cs + i);
-                        const float a = lo[i], b = hi[i];
+                        const float a = lo[i] * rs, b = hi[i] * rs;
                         lo[i] = a * t.x - b * t.y;
                         hi[i] = b * t.x + a * t.y;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        lo[i] *= rs;
+                        hi[i] *= rs;
                     }
                 }
                 store_bf16x32(orow + col0 + j * 32, lo);
@@ -189,6 +206,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t trow
         __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<size_t>(row_ok ? row : 0) * p.ldo +
                               static_cast<size_t>(n_idx) * (BN / 2);
         if (n0 < p.N) {
+            const float rs = row_rstd(p, row, row_ok);
 #pragma unroll 1
             for (int c = 0; c < BN / 64; ++c) {
                 float g[32], u[32];
@@ -196,7 +214,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t trow
                 load_acc(trow + BN / 2 + c * 32, u);
                 if (!row_ok) continue;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) g[i] = silu_f(g[i]) * u[i];
+                for (int i = 0; i < 32; ++i) g[i] = silu_f(g[i] * rs) * (u[i] * rs);
                 store_bf16x32(orow + c * 32, g);
             }
         }
@@ -209,10 +227,18 @@ constexpr int EPI_STAGE_BYTES = 4 * 32 * 32 * 4;  // pair kernel: one 32 x 32 fp
 // row per lane) is transposed through a swizzled shared-memory block so that eight lanes cover the 128
 // contiguous bytes of one residual row.  `row0` is the first row of the warp's 32, `stage` its block.
 __device__ __forceinline__ void epilogue_resid_staged(const GemmParams& p, uint32_t trow, int row0, int n0, int lane,
-                                                      float4* stage) {
+                                                      float4* stage, int n_idx, int n_tiles) {
     const int n_chunks = min(BN, p.N - n0) / 32;
     const int sub = lane >> 3, c4 = lane & 7;
     float* gbase = reinterpret_cast<float*>(p.out) + static_cast<size_t>(row0) * p.ldo + n0 + c4 * 4;
+    // folded RMSNorm of the stream just updated: bf16(x * gain) beside it, and per row the sum of squares of
+    // this tile's columns (lanes that share a row combine theirs at the end)
+    const bool norm = p.norm_gain != nullptr;
+    const __nv_bfloat16* gain = reinterpret_cast<const __nv_bfloat16*>(p.norm_gain) + n0 + c4 * 4;
+    __nv_bfloat16* xg = reinterpret_cast<__nv_bfloat16*>(p.xg_out) + static_cast<size_t>(row0) * p.N + n0 + c4 * 4;
+    float ssq[8];
+#pragma unroll
+    for (int it = 0; it < 8; ++it) ssq[it] = 0.f;
     float4 nxt[8];
     auto fetch = [&](int c, float4 (&dst)[8]) {
 #pragma unroll
@@ -234,6 +260,11 @@ __device__ __forceinline__ void epilogue_resid_staged(const GemmParams& p, uint3
         for (int i = 0; i < 8; ++i)
             stage[lane * 8 + (i ^ (lane & 7))] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
         __syncwarp();
+        float g0 = 0.f, g1 = 0.f, g2 = 0.f, g3 = 0.f;
+        if (norm) {
+            const uint2 gv = __ldg(reinterpret_cast<const uint2*>(gain + c * 32));
+            g0 = bf16_lo(gv.x); g1 = bf16_hi(gv.x); g2 = bf16_lo(gv.y); g3 = bf16_hi(gv.y);
+        }
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
             const int r = it * 4 + sub;
@@ -242,9 +273,27 @@ __device__ __forceinline__ void epilogue_resid_staged(const GemmParams& p, uint3
                 float4 x = cur[it];
                 x.x += a.x; x.y += a.y; x.z += a.z; x.w += a.w;
                 *reinterpret_cast<float4*>(gbase + static_cast<size_t>(r) * p.ldo + c * 32) = x;
+                if (norm) {
+                    ssq[it] += (x.x * x.x + x.y * x.y) + (x.z * x.z + x.w * x.w);
+                    uint2 o;
+                    o.x = pack_bf16(x.x * g0, x.y * g1);
+                    o.y = pack_bf16(x.z * g2, x.w * g3);
+                    *reinterpret_cast<uint2*>(xg + static_cast<size_t>(r) * p.N + c * 32) = o;
+                }
             }
         }
         __syncwarp();
+    }
+    if (norm) {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            float s = ssq[it];
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, 1);
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, 2);
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, 4);
+            const int r = it * 4 + sub;
+            if (c4 == 0 && row0 + r < p.M) p.sumsq_out[static_cast<size_t>(row0 + r) * n_tiles + n_idx] = s;
+        }
     }
 }
 
@@ -621,7 +670,7 @@ gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             const uint32_t trow = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
             if constexpr (EPI == EPI_RESID_ADD || EPI == EPI_RESID_ADD_COMPARE) {
                 float4* stage = reinterpret_cast<float4*>(smem_raw + (base - raw) + P_TILE_BYTES + BAR_BYTES) + quarter * 256;
-                epilogue_resid_staged(p, trow, row - lane, n0, lane, stage);
+                epilogue_resid_staged(p, trow, row - lane, n0, lane, stage, tc.n_idx, num_n);
             } else {
                 epilogue_tile<EPI>(p, trow, row, n0, tc.n_idx);
             }

@@ -44,6 +44,17 @@ struct GemmParams {
     float* partials;        // [n_check][n_tiles_n][kNPart]
     float* hidden_out;      // optional [n_check][N]
     CmpParams cmp;
+    // RMSNorm folded into the neighbouring projections (x * rsqrt(mean x^2 + eps) * gain = rstd * (x * gain)).
+    // Producer, EPI_RESID_ADD(_COMPARE) of the CTA-pair kernel: with norm_gain set, the epilogue also writes
+    // xg_out[M][N] = bf16(residual * gain) and sumsq_out[M][n_tiles] = sum of squares of its row segment.
+    const void* norm_gain;  // bf16 [N]
+    void* xg_out;           // bf16 [M][N]
+    float* sumsq_out;       // [M][ceil(N / 256)]
+    // Consumer, EPI_QKV_ROPE and EPI_SWIGLU: with sumsq_in set, row m of the accumulator is multiplied by
+    // rsqrt(sum_k sumsq_in[m][k] * norm_inv_d + norm_eps) (parts added in index order) before the epilogue proper.
+    const float* sumsq_in;  // [M][n_parts]
+    int n_parts;
+    float norm_eps, norm_inv_d;
     int* status;
 };
 
@@ -71,6 +82,10 @@ cudaError_t launch_embed(const int* tokens, const void* table, int n_tokens, int
 // resid[n] (fp32) = recorded states in `dtype` (VERILLM_BF16 / VERILLM_F32): input of a segment-local pass
 cudaError_t launch_load_states(const void* src, int dtype, size_t n, float* resid, cudaStream_t stream);
 cudaError_t launch_rmsnorm(const float* x, const void* gain, void* y, int rows, int d, float eps,
+                           cudaStream_t stream);
+// The producer half of a folded norm as a kernel of its own (first layer of a pass, small batches):
+// y = bf16(x * gain), sumsq[row][0] = sum of squares of the row, sumsq[row][1 .. n_parts) = 0.
+cudaError_t launch_prenorm(const float* x, const void* gain, void* y, float* sumsq, int n_parts, int rows, int d,
                            cudaStream_t stream);
 cudaError_t launch_compare_rows(const float* hidden, const void* committed, int n_rows, int d, const CmpParams& cmp,
                                 float* partials, cudaStream_t stream);

@@ -75,6 +75,7 @@ struct verillm_model {
     int *pos_of_token = nullptr, *seq_of_token = nullptr, *slot_first = nullptr, *slot_next = nullptr;
     int *tok_of_slot = nullptr, *seq_of_slot = nullptr, *cu_dev = nullptr, *status = nullptr;
     float* partials = nullptr;
+    float* sumsq = nullptr;  // [max_tokens][n_tiles_d]: per-tile sums of squares of the residual rows (folded RMSNorm)
     float2* rope_cs = nullptr;
     CUtensorMap t_xn, t_attn, t_mid;
     CUtensorMap t_qkv_q, t_qkv_kv;  // attention operands: boxes of 128 query rows / 64 key rows
@@ -189,13 +190,20 @@ int check_slots(const verillm_model* m, const int32_t* cu, int32_t batch, const 
 
 // One transformer block over M packed tokens, residual stream updated in place.  With cmp_layer set the
 // down projection runs the gather(-and-compare) epilogue.
+//
+// Both RMSNorms are folded into the projections around them: the producer of the residual stream (the O and
+// down projections, or a small kernel at the start of a pass and for batches the single-CTA GEMM serves) leaves
+// bf16(x * gain) in `xn` and the rows' sums of squares in `sumsq`; the consumer (QKV, gate/up) multiplies its
+// accumulator rows by rsqrt(mean x^2 + eps).
 struct LayerRun {
     int M, batch, max_len;
     const int* cu_dev;
     const GemmParams* cmp_layer;  // fields slot_first .. cmp, or nullptr
+    int next_layer;               // layer whose attention norm follows this block's output, -1 if none
+    bool norm_ready;              // in/out: xn / sumsq already hold the input of this layer's attention norm
 };
 
-int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStream_t st, int* launches) {
+int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st, int* launches) {
     const verillm_config& c = m->cfg;
     const LayerDev& w = m->layers[l];
     GemmParams p;
@@ -206,11 +214,22 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
     // Tile walk in bands of 16 tile-rows for every projection (measured: bands of 4, 8, 32 and "all rows" are
     // no faster, also for the K = d_model projections whose activations would fit in L2).
     const int band_d = 16;
+    const bool fold = p.pair != 0;  // the coalesced residual epilogue of the CTA-pair kernel carries the producer half
+    auto consumer = [&](GemmParams& q) {
+        q.sumsq_in = m->sumsq; q.n_parts = m->n_tiles_d; q.norm_eps = c.rms_eps; q.norm_inv_d = 1.f / static_cast<float>(c.d_model);
+    };
+    auto producer = [&](GemmParams& q, const void* gain) {
+        q.norm_gain = gain; q.xg_out = gain ? m->xn : nullptr; q.sumsq_out = gain ? m->sumsq : nullptr;
+    };
 
-    CU_TRY(launch_rmsnorm(m->resid, w.attn_norm, m->xn, r.M, c.d_model, c.rms_eps, st));
-    prof_mark(m, VERILLM_PROF_RMSNORM, st);
+    if (!r.norm_ready) {
+        CU_TRY(launch_prenorm(m->resid, w.attn_norm, m->xn, m->sumsq, m->n_tiles_d, r.M, c.d_model, st));
+        prof_mark(m, VERILLM_PROF_RMSNORM, st);
+        *launches += 1;
+    }
     p.N = m->n_qkv; p.K = c.d_model; p.out = m->qkv; p.ldo = m->n_qkv; p.group_m = band_d;
     p.rope_cs = m->rope_cs; p.pos_of_token = m->pos_of_token; p.head_dim = c.head_dim; p.rope_cols = m->d_q + m->d_kv;
+    consumer(p);
     CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, p.pair ? w.t_wqkv_h : w.t_wqkv, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_QKV, st);
     CU_TRY(launch_attention_tc(m->t_qkv_q, m->t_qkv_kv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads,
@@ -218,15 +237,25 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
     prof_mark(m, VERILLM_PROF_ATTENTION, st);
     p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
     p.group_m = band_d;
+    p.sumsq_in = nullptr;
+    producer(p, fold ? w.ffn_norm : nullptr);
     CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_attn, p.pair ? w.t_wo_h : w.t_wo, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_O, st);
-    CU_TRY(launch_rmsnorm(m->resid, w.ffn_norm, m->xn, r.M, c.d_model, c.rms_eps, st));
-    prof_mark(m, VERILLM_PROF_RMSNORM, st);
+    if (!fold) {
+        CU_TRY(launch_prenorm(m->resid, w.ffn_norm, m->xn, m->sumsq, m->n_tiles_d, r.M, c.d_model, st));
+        prof_mark(m, VERILLM_PROF_RMSNORM, st);
+        *launches += 1;
+    }
     p.N = 2 * c.d_ffn; p.K = c.d_model; p.out = m->mid; p.ldo = c.d_ffn; p.group_m = band_d;
+    producer(p, nullptr);
+    consumer(p);
     CU_TRY(launch_gemm(EPI_SWIGLU, m->t_xn, p.pair ? w.t_wgu_h : w.t_wgu, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_GATE_UP, st);
     p.N = c.d_model; p.K = c.d_ffn; p.out = m->resid; p.ldo = c.d_model;
     p.group_m = band_d;
+    p.sumsq_in = nullptr;
+    const bool feeds_next = fold && r.next_layer >= 0;
+    producer(p, feeds_next ? m->layers[r.next_layer].attn_norm : nullptr);
     if (r.cmp_layer) {
         p.slot_first = r.cmp_layer->slot_first; p.slot_next = r.cmp_layer->slot_next; p.n_check = r.cmp_layer->n_check;
         p.committed = r.cmp_layer->committed; p.partials = r.cmp_layer->partials; p.hidden_out = r.cmp_layer->hidden_out;
@@ -236,7 +265,8 @@ int run_layer(verillm_model* m, int l, const LayerRun& r, int* status, cudaStrea
         CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_mid, p.pair ? w.t_wd_h : w.t_wd, p, m->num_sms, st));
     }
     prof_mark(m, VERILLM_PROF_GEMM_DOWN, st);
-    *launches += 7;
+    r.norm_ready = feeds_next;
+    *launches += 5;
     return VERILLM_OK;
 }
 
@@ -297,7 +327,7 @@ void verillm_free(verillm_model* m) {
     cudaFree(m->resid); cudaFree(m->xn); cudaFree(m->qkv); cudaFree(m->attn); cudaFree(m->mid);
     cudaFree(m->pos_of_token); cudaFree(m->seq_of_token); cudaFree(m->slot_first); cudaFree(m->slot_next);
     cudaFree(m->tok_of_slot); cudaFree(m->seq_of_slot); cudaFree(m->cu_dev); cudaFree(m->status);
-    cudaFree(m->partials); cudaFree(m->rope_cs);
+    cudaFree(m->partials); cudaFree(m->sumsq); cudaFree(m->rope_cs);
     cudaFree(m->lm_head); cudaFree(m->tm_y); cudaFree(m->tm_rec); cudaFree(m->tm_claimed);
     DecodeState& d = m->dec;
     cudaFree(d.kv_cache); cudaFree(d.hidden_tmp); cudaFree(d.resid); cudaFree(d.qkv); cudaFree(d.gu);
@@ -423,6 +453,7 @@ int verillm_load_weights(const verillm_config* cfg, const verillm_weights* weigh
     TRY_RC(dev_alloc(&m->cu_dev, static_cast<size_t>(c.max_batch) + 1));
     TRY_RC(dev_alloc(&m->status, 1));
     TRY_RC(dev_alloc(&m->partials, static_cast<size_t>(c.n_layers) * NC * m->n_tiles_d * kNPart));
+    TRY_RC(dev_alloc(&m->sumsq, T * m->n_tiles_d));
     TRY_RC(dev_alloc(&m->rope_cs, T * (c.head_dim / 2)));
 
     // Rows past a call's last token are never stored, but tiles that straddle the end are read: keep them finite.
@@ -526,8 +557,9 @@ static int verify_impl(verillm_model* m, const int32_t* tokens, const void* stat
     std::memset(&cl, 0, sizeof(cl));
     cl.slot_first = m->slot_first; cl.slot_next = m->slot_next; cl.n_check = n_check;
     cl.cmp = cmp_params(*tol, commit_dtype);
-    LayerRun run{M, batch, max_len, m->cu_dev, n_check > 0 ? &cl : nullptr};
+    LayerRun run{M, batch, max_len, m->cu_dev, n_check > 0 ? &cl : nullptr, -1, false};
     for (int l = l0; l < l1; ++l) {
+        run.next_layer = l + 1 < l1 ? l + 1 : -1;
         const size_t slab = static_cast<size_t>(l - l0) * n_check;
         cl.committed = reinterpret_cast<const char*>(committed_hidden) + slab * c.d_model * e_commit;
         cl.partials = m->partials + slab * m->n_tiles_d * kNPart;
@@ -785,9 +817,10 @@ int verillm_decode_commit(verillm_model* m, const int32_t* tokens, const int32_t
         std::memset(&cl, 0, sizeof(cl));
         cl.slot_first = m->slot_first; cl.slot_next = m->slot_next; cl.n_check = n_check;
         cl.committed = nullptr; cl.partials = nullptr;
-        LayerRun run{Mp, batch, max_np, m->cu_dev, n_check > 0 ? &cl : nullptr};
+        LayerRun run{Mp, batch, max_np, m->cu_dev, n_check > 0 ? &cl : nullptr, -1, false};
         int launches = 0;
         for (int l = 0; l < c.n_layers; ++l) {
+            run.next_layer = l + 1 < c.n_layers ? l + 1 : -1;
             cl.hidden_out = d.hidden_tmp + static_cast<size_t>(l) * n_check * c.d_model;
             if ((rc = run_layer(m, l, run, dev_status, st, &launches))) return rc;
             // run_layer leaves this layer's rotated keys and values in qkv: append them to the cache

@@ -57,7 +57,7 @@ def test_llama8b_full_depth_sampled_positions_and_honest_trace():
     rep = model.verify_prefill(flat, cu, committed, cs, cp, want_hidden=True)
     torch.cuda.synchronize()
     g = rep.cpu()
-    assert g["status"] == 0 and model.last_launch_count() == 3 + 7 * 32 + 2
+    assert g["status"] == 0 and model.last_launch_count() == 3 + 1 + 5 * 32 + 2
 
     # --- sampled outputs against the oracle
     stats_o = np.transpose(vo.compare_stats(pre.hidden, comm_sampled.to(torch.float64).numpy(), "bf16", vo.Tol()), (1, 0, 2))
