@@ -227,13 +227,13 @@ constexpr int EPI_STAGE_BYTES = 4 * 32 * 32 * 4;  // pair kernel: one 32 x 32 fp
 // row per lane) is transposed through a swizzled shared-memory block so that eight lanes cover the 128
 // contiguous bytes of one residual row.  `row0` is the first row of the warp's 32, `stage` its block.
 __device__ __forceinline__ void epilogue_resid_staged(const GemmParams& p, uint32_t trow, int row0, int n0, int lane,
-                                                      float4* stage, int n_idx, int n_tiles) {
+                                                      float4* stage, int n_idx, int n_tiles, bool final_part) {
     const int n_chunks = min(BN, p.N - n0) / 32;
     const int sub = lane >> 3, c4 = lane & 7;
     float* gbase = reinterpret_cast<float*>(p.out) + static_cast<size_t>(row0) * p.ldo + n0 + c4 * 4;
     // folded RMSNorm of the stream just updated: bf16(x * gain) beside it, and per row the sum of squares of
     // this tile's columns (lanes that share a row combine theirs at the end)
-    const bool norm = p.norm_gain != nullptr;
+    const bool norm = p.norm_gain != nullptr && final_part;  // only the last K part of a tile holds final values
     const __nv_bfloat16* gain = reinterpret_cast<const __nv_bfloat16*>(p.norm_gain) + n0 + c4 * 4;
     __nv_bfloat16* xg = reinterpret_cast<__nv_bfloat16*>(p.xg_out) + static_cast<size_t>(row0) * p.N + n0 + c4 * 4;
     float ssq[8];
@@ -244,7 +244,8 @@ __device__ __forceinline__ void epilogue_resid_staged(const GemmParams& p, uint3
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
             const int r = it * 4 + sub;
-            if (row0 + r < p.M) dst[it] = *reinterpret_cast<const float4*>(gbase + static_cast<size_t>(r) * p.ldo + c * 32);
+            // (read around L1: another SM may have added an earlier K part of this tile)
+            if (row0 + r < p.M) dst[it] = __ldcg(reinterpret_cast<const float4*>(gbase + static_cast<size_t>(r) * p.ldo + c * 32));
         }
     };
     if (n_chunks > 0) fetch(0, nxt);
@@ -530,6 +531,60 @@ constexpr int P_STAGE_BYTES = A_STAGE_BYTES + P_B_STAGE_BYTES;
 constexpr int P_TILE_BYTES = P_STAGES * P_STAGE_BYTES;
 constexpr int P_GEMM_SMEM = P_TILE_BYTES + BAR_BYTES + EPI_STAGE_BYTES + 1024;
 
+// Bounded wait until a global counter has reached `target` (written with atomicAdd by other CTAs of this launch).
+__device__ __forceinline__ bool wait_counter(const int* counter, int target, int* status) {
+    const volatile int* c = counter;
+    const long long t0 = clock64();
+    while (*c < target) {
+        if (clock64() - t0 > kWaitLimitCycles) {
+            if (status) atomicCAS(status, 0, VERILLM_DEV_WAIT_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+
+// Work of one CTA pair.  Tiles are dealt round robin over `pairs_total` pairs; the last, partly filled round
+// of a projection whose epilogue is additive (residual += accumulator) is cut along K into `split` parts so
+// that it occupies all pairs: part q of a tile adds its partial product to the residual after part q-1 has
+// (a per-tile counter in global memory orders them, so the sum is formed in a fixed order), and only the
+// last part runs what needs the final values (folded norm, gather-and-compare).
+struct SplitPlan {
+    int full, rem, split;
+};
+__host__ __device__ inline SplitPlan split_plan(int num_tiles, int pairs_total, int num_kb, bool additive) {
+    SplitPlan s;
+    s.full = num_tiles / pairs_total;
+    s.rem = num_tiles % pairs_total;
+    s.split = 1;
+    if (additive && s.rem > 0) {
+        int sp = pairs_total / s.rem;
+        if (sp > 4) sp = 4;
+        if (sp > num_kb / 16) sp = num_kb / 16;  // parts of at least 16 K steps
+        if (sp > 1) s.split = sp;
+    }
+    return s;
+}
+struct PairItem {
+    int tile, kb0, kb1, part, n_parts, rem_idx;
+};
+// k-th item of pair x; false past the end.
+__device__ __forceinline__ bool pair_item(const SplitPlan& s, int pairs_total, int num_kb, int x, int k, PairItem& it) {
+    it.kb0 = 0; it.kb1 = num_kb; it.part = 0; it.n_parts = 1; it.rem_idx = -1;
+    if (k < s.full) {
+        it.tile = x + k * pairs_total;
+        return true;
+    }
+    if (k > s.full || x >= s.rem * s.split) return false;
+    it.rem_idx = x % s.rem;
+    it.part = x / s.rem;
+    it.n_parts = s.split;
+    it.tile = s.full * pairs_total + it.rem_idx;
+    it.kb0 = it.part * num_kb / s.split;
+    it.kb1 = (it.part + 1) * num_kb / s.split;
+    return true;
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -553,12 +608,14 @@ gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();  // 0: leader (issues the MMAs), 1: peer
     const int pair_id = blockIdx.x >> 1;
-    const int num_pairs = gridDim.x >> 1;
     const int num_m = (p.M + 2 * BM - 1) / (2 * BM);  // tile-rows of 256
     const int num_n = (p.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     const int num_kb = (p.K + BK - 1) / BK;
     const int group_m = p.group_m > 0 ? p.group_m : 8;
+    constexpr bool kAdditive = EPI == EPI_RESID_ADD || EPI == EPI_RESID_ADD_COMPARE;
+    const SplitPlan plan = split_plan(num_tiles, p.pairs_total, num_kb, kAdditive && p.split_flags != nullptr);
+    PairItem item;
 
     if (threadIdx.x == 0) {
         s_failed = 0;
@@ -591,11 +648,11 @@ gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
-                const TileCoord tc = tile_coord(tile, num_m, num_n, group_m);
+            for (int k = 0; ok && pair_item(plan, p.pairs_total, num_kb, pair_id, k, item); ++k) {
+                const TileCoord tc = tile_coord(item.tile, num_m, num_n, group_m);
                 const int a_row = tc.m_idx * 2 * BM + static_cast<int>(rank) * BM;
                 const int b_row = tc.n_idx * BN + static_cast<int>(rank) * 128;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = item.kb0; kb < item.kb1; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status)) {
                         ok = false;
                         break;
@@ -621,14 +678,14 @@ gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
-            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
+            for (int k = 0; ok && pair_item(plan, p.pairs_total, num_kb, pair_id, k, item); ++k) {
                 if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, p.status)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = item.kb0; kb < item.kb1; ++kb) {
                     if (!mbar_wait(full_bar(stage), phase, p.status)) {
                         ok = false;
                         break;
@@ -637,8 +694,8 @@ gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                     const uint64_t a_desc = umma_desc_k_sw128(a_base + stage * A_STAGE_BYTES);
                     const uint64_t b_desc = umma_desc_k_sw128(b_base + stage * P_B_STAGE_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k)
-                        umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    for (int kk = 0; kk < BK / UMMA_K; ++kk)
+                        umma_bf16_pair(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, idesc, (kb != item.kb0 || kk != 0) ? 1u : 0u);
                     umma_commit_pair(empty_bar(stage));  // frees the stage in both CTAs
                     if (++stage == P_STAGES) {
                         stage = 0;
@@ -658,8 +715,8 @@ gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
-            const TileCoord tc = tile_coord(tile, num_m, num_n, group_m);
+        for (int k = 0; ok && pair_item(plan, p.pairs_total, num_kb, pair_id, k, item); ++k) {
+            const TileCoord tc = tile_coord(item.tile, num_m, num_n, group_m);
             if (!mbar_wait(acc_full_bar(acc), acc_phase, p.status)) {
                 ok = false;
                 break;
@@ -668,17 +725,35 @@ gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             const int row = tc.m_idx * 2 * BM + static_cast<int>(rank) * BM + quarter * 32 + lane;
             const int n0 = tc.n_idx * BN;
             const uint32_t trow = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
-            if constexpr (EPI == EPI_RESID_ADD || EPI == EPI_RESID_ADD_COMPARE) {
+            const bool final_part = item.part == item.n_parts - 1;
+            if constexpr (kAdditive) {
+                if (item.part > 0) {
+                    // the earlier parts of this tile (eight epilogue warps each) must have added theirs
+                    uint32_t done = 1u;
+                    if (lane == 0) done = wait_counter(p.split_flags + item.rem_idx, 8 * item.part, p.status) ? 1u : 0u;
+                    if (__shfl_sync(0xFFFFFFFFu, done, 0) == 0u) {
+                        ok = false;
+                        break;
+                    }
+                    __threadfence();
+                }
                 float4* stage = reinterpret_cast<float4*>(smem_raw + (base - raw) + P_TILE_BYTES + BAR_BYTES) + quarter * 256;
-                epilogue_resid_staged(p, trow, row - lane, n0, lane, stage, tc.n_idx, num_n);
+                epilogue_resid_staged(p, trow, row - lane, n0, lane, stage, tc.n_idx, num_n, final_part);
             } else {
                 epilogue_tile<EPI>(p, trow, row, n0, tc.n_idx);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(acc), 0));  // the leader collects all 8
+            if constexpr (kAdditive) {
+                if (!final_part) {  // publish this warp's share of the partial sum
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) atomicAdd(p.split_flags + item.rem_idx, 1);
+                }
+            }
             if constexpr (EPI == EPI_RESID_ADD_COMPARE) {
-                if (row < p.M && p.slot_first != nullptr) compare_row(p, row, n0, tc.n_idx, num_n);
+                if (final_part && row < p.M && p.slot_first != nullptr) compare_row(p, row, n0, tc.n_idx, num_n);
                 __syncwarp();
             }
             acc ^= 1;
@@ -710,8 +785,17 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
                         cudaStream_t stream) {
     const int num_tiles = ((p.M + 2 * BM - 1) / (2 * BM)) * ((p.N + BN - 1) / BN);
     if (num_tiles <= 0) return cudaSuccess;
-    int pairs = num_sms / 2;
-    if (num_tiles < pairs) pairs = num_tiles;
+    GemmParams q = p;
+    q.pairs_total = num_sms / 2;
+    constexpr bool additive = EPI == EPI_RESID_ADD || EPI == EPI_RESID_ADD_COMPARE;
+    const SplitPlan plan = split_plan(num_tiles, q.pairs_total, (p.K + BK - 1) / BK, additive && p.split_flags != nullptr);
+    if (plan.split > 1) {  // the per-tile part counters of the last round start at zero
+        const cudaError_t e = cudaMemsetAsync(p.split_flags, 0, sizeof(int) * plan.rem, stream);
+        if (e != cudaSuccess) return e;
+    } else {
+        q.split_flags = nullptr;
+    }
+    const int pairs = plan.full > 0 ? q.pairs_total : plan.rem * plan.split;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs);
     cfg.blockDim = dim3(GEMM_THREADS);
@@ -724,7 +808,7 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_bf16_tcgen05_pair<EPI>, ta, tb, p);
+    return cudaLaunchKernelEx(&cfg, gemm_bf16_tcgen05_pair<EPI>, ta, tb, q);
 }
 
 template <int EPI>

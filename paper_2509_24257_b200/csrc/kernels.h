@@ -55,6 +55,10 @@ struct GemmParams {
     const float* sumsq_in;  // [M][n_parts]
     int n_parts;
     float norm_eps, norm_inv_d;
+    // CTA-pair kernel with an additive epilogue: per-tile counters (one int per pair of SMs) that order the K
+    // parts of the last, partly filled round of tiles; nullptr: no K split.  pairs_total is set by the launcher.
+    int* split_flags;
+    int pairs_total;
     int* status;
 };
 

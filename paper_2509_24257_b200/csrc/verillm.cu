@@ -75,6 +75,7 @@ struct verillm_model {
     int *pos_of_token = nullptr, *seq_of_token = nullptr, *slot_first = nullptr, *slot_next = nullptr;
     int *tok_of_slot = nullptr, *seq_of_slot = nullptr, *cu_dev = nullptr, *status = nullptr;
     float* partials = nullptr;
+    int* split_flags = nullptr;  // K-part counters of the GEMMs' last round (one per pair of SMs)
     float* sumsq = nullptr;  // [max_tokens][n_tiles_d]: per-tile sums of squares of the residual rows (folded RMSNorm)
     float2* rope_cs = nullptr;
     CUtensorMap t_xn, t_attn, t_mid;
@@ -238,6 +239,7 @@ int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st
     p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
     p.group_m = band_d;
     p.sumsq_in = nullptr;
+    p.split_flags = m->split_flags;
     producer(p, fold ? w.ffn_norm : nullptr);
     CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_attn, p.pair ? w.t_wo_h : w.t_wo, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_O, st);
@@ -247,6 +249,7 @@ int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st
         *launches += 1;
     }
     p.N = 2 * c.d_ffn; p.K = c.d_model; p.out = m->mid; p.ldo = c.d_ffn; p.group_m = band_d;
+    p.split_flags = nullptr;
     producer(p, nullptr);
     consumer(p);
     CU_TRY(launch_gemm(EPI_SWIGLU, m->t_xn, p.pair ? w.t_wgu_h : w.t_wgu, p, m->num_sms, st));
@@ -254,6 +257,7 @@ int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st
     p.N = c.d_model; p.K = c.d_ffn; p.out = m->resid; p.ldo = c.d_model;
     p.group_m = band_d;
     p.sumsq_in = nullptr;
+    p.split_flags = m->split_flags;
     const bool feeds_next = fold && r.next_layer >= 0;
     producer(p, feeds_next ? m->layers[r.next_layer].attn_norm : nullptr);
     if (r.cmp_layer) {
@@ -327,7 +331,7 @@ void verillm_free(verillm_model* m) {
     cudaFree(m->resid); cudaFree(m->xn); cudaFree(m->qkv); cudaFree(m->attn); cudaFree(m->mid);
     cudaFree(m->pos_of_token); cudaFree(m->seq_of_token); cudaFree(m->slot_first); cudaFree(m->slot_next);
     cudaFree(m->tok_of_slot); cudaFree(m->seq_of_slot); cudaFree(m->cu_dev); cudaFree(m->status);
-    cudaFree(m->partials); cudaFree(m->sumsq); cudaFree(m->rope_cs);
+    cudaFree(m->partials); cudaFree(m->sumsq); cudaFree(m->split_flags); cudaFree(m->rope_cs);
     cudaFree(m->lm_head); cudaFree(m->tm_y); cudaFree(m->tm_rec); cudaFree(m->tm_claimed);
     DecodeState& d = m->dec;
     cudaFree(d.kv_cache); cudaFree(d.hidden_tmp); cudaFree(d.resid); cudaFree(d.qkv); cudaFree(d.gu);
@@ -454,6 +458,8 @@ int verillm_load_weights(const verillm_config* cfg, const verillm_weights* weigh
     TRY_RC(dev_alloc(&m->status, 1));
     TRY_RC(dev_alloc(&m->partials, static_cast<size_t>(c.n_layers) * NC * m->n_tiles_d * kNPart));
     TRY_RC(dev_alloc(&m->sumsq, T * m->n_tiles_d));
+    TRY_RC(dev_alloc(&m->split_flags, 256));
+    cudaMemset(m->split_flags, 0, 256 * sizeof(int));
     TRY_RC(dev_alloc(&m->rope_cs, T * (c.head_dim / 2)));
 
     // Rows past a call's last token are never stored, but tiles that straddle the end are read: keep them finite.
