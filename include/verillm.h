@@ -13,7 +13,17 @@
  *    and one workspace sized at load time from max_tokens / max_checks / max_batch.
  *  - All calls enqueue work on the given stream and return without synchronising unless stated;
  *    results are valid once the caller has synchronised the stream.  Host arrays passed to a call
- *    may be reused as soon as the call returns.
+ *    may be reused as soon as the call returns, whether they are pageable or pinned: the library
+ *    copies them into memory of its own before it queues the transfer.
+ *  - A handle serves one call at a time: its workspace, staging arrays and counters are shared by
+ *    all calls, so calls on one handle must not overlap, neither from several threads nor on several
+ *    streams.  Different handles are independent.
+ *  - The projections over more than 128 rows split the last, partly filled round of output tiles
+ *    along K over otherwise idle SM pairs, and a later part waits for the earlier part of the same
+ *    tile, which runs on another SM pair of the same launch.  The parts are dealt so that a part
+ *    never waits for a pair with a higher index, and the wait is bounded: if the GPU is shared with
+ *    other kernels to the point that the producing pair is not scheduled within about two seconds,
+ *    the call ends with VERILLM_DEV_WAIT_TIMEOUT in the status word instead of hanging.
  *  - Return value: 0 on success, a negative VERILLM_E_* code otherwise; nothing is launched when
  *    an argument is rejected.  Problems only the device can see (a token id >= vocab) clamp the
  *    offending index, set *report.status to a positive VERILLM_DEV_* code and force a reject.
@@ -160,15 +170,18 @@ int verillm_verify_prefill(verillm_model *model, const int32_t *tokens, const in
                            const int32_t *check_pos, int32_t n_check, const verillm_tol *tol,
                            const verillm_report *report, void *cuda_stream);
 
-/* Segment-local verification ("for segment i, the verifier uses the recorded upstream hidden states as its inputs
- * and executes only its own block of layers"; T_verify ~ T_prefill / L): blocks layer_begin .. layer_end-1 are
- * recomputed for all positions from the recorded states entering block layer_begin, and compared at the checked
- * positions with the committed outputs of those blocks.
+/* Segment-local verification (Verification Scheme, segment-local recompute; T_verify ~ T_prefill / L): blocks
+ * layer_begin .. layer_end-1 are recomputed for all positions from the recorded states entering block
+ * layer_begin, and compared at the checked positions with the committed outputs of those blocks.
  *  input_states     DEVICE [cu_seqlens[batch]][d_model] in input_dtype (BF16 / F32): the residual stream entering
  *                   block layer_begin at every position (the output of block layer_begin-1, or the embeddings)
  *  committed_hidden DEVICE [layer_end - layer_begin][n_check][d_model]
  * The report arrays have layer_end - layer_begin layers and their layer indices count from layer_begin; all else
- * as verillm_verify_prefill.  Extra errors: E_RANGE for an empty or out-of-range layer interval. */
+ * as verillm_verify_prefill.  Extra errors: E_RANGE for an empty or out-of-range layer interval.
+ * The recorded states come from another party: an entry that is NaN, infinite or beyond 1e15 in magnitude is
+ * read as 0 and its sequence is rejected as a whole (seq_ok = 0, every checked position of it pos_ok = 0 with
+ * first_bad_layer = 0), as an exact recomputation would: one such entry makes every state of its sequence
+ * non-finite.  The other sequences of the batch are unaffected. */
 int verillm_verify_segment(verillm_model *model, const void *input_states, int32_t input_dtype, int32_t layer_begin,
                            int32_t layer_end, const int32_t *cu_seqlens, int32_t batch, const void *committed_hidden,
                            int32_t commit_dtype, const int32_t *check_seq, const int32_t *check_pos, int32_t n_check,
@@ -184,8 +197,8 @@ int verillm_decode_commit(verillm_model *model, const int32_t *tokens, const int
                           int32_t n_prefill, const int32_t *check_seq, const int32_t *check_pos, int32_t n_check,
                           void *committed_out, int32_t commit_dtype, int32_t *status, void *cuda_stream);
 
-/* Tail token check ("TokenMatch(argmax f_LM(S_{L+1}), y) = 1"; token-state cross-check of the forged-output
- * analysis): the last-layer states at the checked positions go through the final RMSNorm and the output
+/* Tail token check (the TokenMatch equation; token-state cross-check of the forged-output analysis): the
+ * last-layer states at the checked positions go through the final RMSNorm and the output
  * head, and the arg-max token of each row is compared with the token the prover claims to have emitted there.
  *  verillm_load_lm_head: output head [vocab][d_model] bf16 (HOST or DEVICE per on_device); the first call also
  *                        allocates the scratch of the check inside the handle.  vocab % 32 == 0 (else E_SHAPE).
@@ -226,7 +239,7 @@ int verillm_compare_noalloc(const float *hidden, const void *committed, int32_t 
                             int32_t n_check, int32_t d_model, const int32_t *check_seq, int32_t batch,
                             const verillm_tol *tol, const verillm_report *report, void *cuda_stream);
 
-/* Relaxed spot check on sampled scalar entries (the on-chain value matching: Delta_j = |v_j - V_j| <= eps,
+/* Relaxed spot check on sampled scalar entries (on-chain value matching: Delta_j = |v_j - V_j| <= eps,
  * agreement rate p_hat = (1/n) sum 1[Delta_j <= eps], positive verdict iff p_hat >= theta).
  *  hidden      DEVICE float32 [n_rows][d_model]: the verifier's states (e.g. one layer of hidden_out)
  *  sample_row / sample_col  HOST int32 [n_samples]: the sampled entries; reference HOST float32 [n_samples]: V_j
@@ -237,7 +250,7 @@ int verillm_spot_check(const float *hidden, int32_t n_rows, int32_t d_model, con
                        const int32_t *sample_col, const float *reference, int32_t n_samples, float eps, float theta,
                        uint8_t *agree_out, float *p_hat_out, uint8_t *verdict_out, void *cuda_stream);
 
-/* Threshold sensitivity of the offline tests ("Threshold Sensitivity Analysis": each threshold is varied while the
+/* Threshold sensitivity of the offline tests (appendix Threshold Sensitivity Analysis: one threshold varies, the
  * others stay at their selected values, and the false-positive / false-negative rates are read off honest and
  * attack traces).  The tests of the verdict are applied to statistics reported by an earlier verify / compare call.
  *  stats      DEVICE float32 [n_cells][VERILLM_NSTAT]: one row per (position, layer) cell, as written to report.stats
@@ -250,8 +263,8 @@ int verillm_spot_check(const float *hidden, int32_t n_rows, int32_t d_model, con
 int verillm_threshold_sweep(const float *stats, const uint8_t *is_attack, int32_t n_cells, const verillm_tol *variants,
                             int32_t n_variants, int32_t *counts_out, void *cuda_stream);
 
-/* Merkle commitment of hidden states ("serializes its output tensor, constructs a Merkle tree over all scalar
- * entries and submits the Merkle root"; canonical float32 leaves, SHA-256): one root per vector.
+/* Merkle commitment of hidden states (Inference Scheme, commitment step: a tree over all scalar entries of the
+ * serialised output tensor, whose root is submitted; canonical float32 leaves, SHA-256): one root per vector.
  *  states    DEVICE float32 [n_vec][d_model]; roots_out DEVICE uint8 [n_vec][32]
  * Leaf j = SHA-256(4 bytes of entry j, little-endian IEEE-754 float32); node = SHA-256(left || right); an odd
  * node at the end of a level is paired with itself; a single entry's leaf is its own root.
@@ -290,6 +303,13 @@ enum {
 };
 int verillm_profile_enable(verillm_model *model, int32_t on);
 int verillm_profile_read(verillm_model *model, float *ms, int32_t *launches);
+
+/* Exercise of the bounded wait that every pipeline of the library uses (failure detection; the paper has no
+ * counterpart): one thread waits, for at most limit_cycles SM clock cycles (1 .. 2e9), on a barrier that nothing
+ * signals, holding no copy in flight and no tensor memory.  *status (DEVICE) receives VERILLM_DEV_WAIT_TIMEOUT and
+ * *gave_up (DEVICE, optional) 1; the context stays usable.  The waits inside the real kernels use the same code
+ * with a limit of about two seconds. */
+int verillm_selftest_wait_timeout(int64_t limit_cycles, int32_t *status, int32_t *gave_up, void *cuda_stream);
 
 void verillm_free(verillm_model *model);
 const char *verillm_strerror(int code);

@@ -31,7 +31,7 @@ EXPORTS = (
     "verillm_op_rmsnorm", "verillm_op_attention", "verillm_free", "verillm_strerror",
     "verillm_last_launch_count", "verillm_profile_enable", "verillm_profile_read",
     "verillm_load_lm_head", "verillm_token_match", "verillm_verify_segment", "verillm_spot_check", "verillm_merkle_roots",
-    "verillm_threshold_sweep",
+    "verillm_threshold_sweep", "verillm_selftest_wait_timeout",
 )
 PROF_CLASSES = ("setup", "rmsnorm", "gemm_qkv_rope", "attention", "gemm_o_resid", "gemm_gate_up_swiglu",
                 "gemm_down_resid_compare", "verdict")
@@ -122,6 +122,8 @@ def lib() -> C.CDLL:
         L.verillm_merkle_roots.restype = C.c_int
         L.verillm_threshold_sweep.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(Tol), C.c_int32, C.c_void_p, C.c_void_p]
         L.verillm_threshold_sweep.restype = C.c_int
+        L.verillm_selftest_wait_timeout.argtypes = [C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.verillm_selftest_wait_timeout.restype = C.c_int
         L.verillm_load_lm_head.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
         L.verillm_load_lm_head.restype = C.c_int
         L.verillm_token_match.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -426,6 +428,18 @@ def threshold_sweep(stats: torch.Tensor, is_attack: torch.Tensor, variants: Sequ
         _check(lib().verillm_threshold_sweep(stats.data_ptr(), is_attack.data_ptr(), stats.shape[0], arr, len(variants),
                                              counts.data_ptr(), _stream_ptr(stream)), "verillm_threshold_sweep")
     return counts
+
+
+def selftest_wait_timeout(limit_cycles: int, device="cuda:0", stream: Optional[torch.cuda.Stream] = None):
+    """Runs the library's bounded wait on a barrier nobody signals.  Returns device tensors (status int32 [1],
+    gave_up int32 [1])."""
+    device = torch.device(device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    gave_up = torch.zeros(1, dtype=torch.int32, device=device)
+    with torch.cuda.device(device):
+        _check(lib().verillm_selftest_wait_timeout(int(limit_cycles), status.data_ptr(), gave_up.data_ptr(),
+                                                   _stream_ptr(stream)), "verillm_selftest_wait_timeout")
+    return status, gave_up
 
 
 def merkle_roots(states: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:

@@ -1,5 +1,5 @@
 // Causal grouped-query attention over packed sequences on the fifth-generation tensor cores:
-// softmax(q k^T / sqrt(dh) + causal mask) v, flash style ("a single forward pass under the causal mask").
+// softmax(q k^T / sqrt(dh) + causal mask) v, flash style (the one causal pass of Full-Sequence Prefill, Eq. 1).
 //
 // A unit of work is 128 query rows of one (sequence, query head), walking the key/value tiles of 64
 // positions up to the diagonal.  CTAs are persistent, two per SM: each takes its share of the units
@@ -192,6 +192,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
+    // up to here only the CTA's own resources and the sequence boundaries (written before the chain of layer
+    // kernels started) were touched: all of it may run under the tail of the projection that produces q, k, v
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp == 5) {
         // ------------------------------------------------------------ TMA producer of keys and values (one thread)
@@ -515,7 +519,7 @@ cudaError_t attention_tc_init() {
 
 cudaError_t launch_attention_tc(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, const int* cu_seqlens_dev,
                                 int batch, int max_seqlen, int n_heads, int n_kv_heads, int head_dim, void* out,
-                                int* status, int num_sms, cudaStream_t stream) {
+                                int* status, int num_sms, int overlap_prologue, cudaStream_t stream) {
     if (batch <= 0 || max_seqlen <= 0) return cudaSuccess;
     const int n_qblocks = (max_seqlen + TC_BM - 1) / TC_BM;
     if (n_heads > 1024 || n_qblocks * (TC_BM / TC_BN) > 2047) return cudaErrorInvalidValue;  // packed work-unit fields
@@ -523,15 +527,26 @@ cudaError_t launch_attention_tc(const CUtensorMap& tmap_q, const CUtensorMap& tm
     const long long units = static_cast<long long>(n_qblocks) * n_heads * batch;
     const dim3 grid(static_cast<unsigned>(units < 2LL * num_sms ? units : 2LL * num_sms));
     __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out);
-    if (head_dim == 64)
-        attn_tc_kernel<64><<<grid, TC_THREADS, TcSmem<64>::TOTAL, stream>>>(tmap_q, tmap_kv, cu_seqlens_dev, batch,
-                                                                           n_qblocks, n_heads, n_kv_heads, o, status);
-    else if (head_dim == 128)
-        attn_tc_kernel<128><<<grid, TC_THREADS, TcSmem<128>::TOTAL, stream>>>(tmap_q, tmap_kv, cu_seqlens_dev, batch,
-                                                                             n_qblocks, n_heads, n_kv_heads, o, status);
-    else
-        return cudaErrorInvalidValue;
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(TC_THREADS);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap_prologue ? 1 : 0;
+    if (head_dim == 64) {
+        cfg.dynamicSmemBytes = TcSmem<64>::TOTAL;
+        return cudaLaunchKernelEx(&cfg, attn_tc_kernel<64>, tmap_q, tmap_kv, cu_seqlens_dev, batch, n_qblocks, n_heads,
+                                  n_kv_heads, o, status);
+    }
+    if (head_dim == 128) {
+        cfg.dynamicSmemBytes = TcSmem<128>::TOTAL;
+        return cudaLaunchKernelEx(&cfg, attn_tc_kernel<128>, tmap_q, tmap_kv, cu_seqlens_dev, batch, n_qblocks, n_heads,
+                                  n_kv_heads, o, status);
+    }
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace vl

@@ -62,21 +62,33 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait on a phase parity.  Returns false (after recording the timeout) if the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+// Bounded wait on a phase parity: gives up after `limit_cycles` SM clock cycles.  Returns false (after
+// recording the timeout in *status) if the limit ran out.
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, int* status, long long limit_cycles) {
 #pragma unroll 1
     for (int i = 0; i < 128; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
 #pragma unroll 1
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > limit_cycles) {
             if (status) atomicCAS(status, 0, VERILLM_DEV_WAIT_TIMEOUT);
             return false;
         }
     }
     return true;
 }
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+    return mbar_wait_limit(bar, parity, status, kWaitLimitCycles);
+}
+
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with programmatic stream serialisation may start while its predecessor in the stream is
+// still running; it must not touch memory the predecessor produces (or still reads) before pdl_wait(), which
+// returns once every earlier kernel of the stream has completed and its writes are visible.  Both are no-ops
+// in a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ---------------------------------------------------------------- TMA (no multicast anywhere)
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {

@@ -41,6 +41,20 @@ inline CmpParams make_cmp_params(int commit_dtype, float tau_large, float e_w, i
     return c;
 }
 
+// packed fp32 pairs: d = a * b + c and d = a + b on both halves in one instruction
+__device__ __forceinline__ float2 cmp_ffma2(float2 a, float2 b, float2 c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;"
+        : "=l"(d)
+        : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)), "l"(reinterpret_cast<uint64_t&>(c)));
+    return reinterpret_cast<float2&>(d);
+}
+__device__ __forceinline__ float2 cmp_fadd2(float2 a, float2 b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)));
+    return reinterpret_cast<float2&>(d);
+}
+
 struct CmpAcc {
     float ss, rr, sa, sg, mx;
     uint32_t n_mis, n_large_m, n_small_w, n_exact, n_qsmall, n_zlarge, n_nonfinite;

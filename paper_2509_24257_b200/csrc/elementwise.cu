@@ -182,14 +182,18 @@ __global__ void compare_rows_kernel(const float* __restrict__ hidden, const void
 // ------------------------------------------------------------------ verdict
 // One warp per check slot, lanes over layers: each lane sums the column-tile partials of its layers in
 // a fixed order, derives the reported statistics and applies the enabled tests (b = 1[T_v <= tau]; a
-// non-finite value or a device-side error rejects); the first failing layer is the minimum over lanes.
+// non-finite value, a device-side error or a sequence marked as malformed rejects); the first failing layer is
+// the minimum over lanes.
 __global__ void verdict_kernel(const float* __restrict__ partials, int n_layers, int n_check, int n_tiles, int d,
-                               TolDev tol, const int* __restrict__ status, float* __restrict__ stats,
+                               TolDev tol, const int* __restrict__ status, const int* __restrict__ seq_of_slot,
+                               const int* __restrict__ seq_flags, float* __restrict__ stats,
                                uint8_t* __restrict__ pos_ok, int* __restrict__ first_bad_layer) {
     const int slot = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (slot >= n_check) return;
-    const bool dev_error = status != nullptr && *status != 0;
+    // a device-side error rejects everything; malformed recorded states reject their sequence
+    const bool dev_error = (status != nullptr && *status != 0) ||
+                           (seq_flags != nullptr && seq_flags[seq_of_slot[slot]] != 0);
     int first_bad = 0x7FFFFFFF;
     const float inv_d = 1.f / static_cast<float>(d);
     for (int l = lane; l < n_layers; l += 32) {
@@ -292,15 +296,19 @@ threshold_sweep_kernel(const float* __restrict__ stats, const uint8_t* __restric
 }
 
 // One block per sequence, threads over check slots: accept iff all its checked positions were accepted (one
-// deviation above tolerance suffices to fail); score = mean MAE over its (slot, layer) cells.  Per-thread
+// deviation above tolerance suffices to fail, and so does a device-side error or malformed input of that
+// sequence); score = mean MAE over its (slot, layer) cells.  Per-thread
 // double sums are combined by a fixed shuffle tree and then in warp order, so the result is reproducible.
 constexpr int kSeqThreads = 1024;
 __global__ void __launch_bounds__(kSeqThreads)
 seq_verdict_kernel(const float* __restrict__ stats, const uint8_t* __restrict__ pos_ok,
                    const int* __restrict__ seq_of_slot, int n_check, int n_layers, int batch,
+                   const int* __restrict__ status, const int* __restrict__ seq_flags,
                    uint8_t* __restrict__ seq_ok, float* __restrict__ seq_score) {
     const int b = blockIdx.x;
-    int bad = 0, cells = 0;
+    // a device-side error invalidates every result of the call, also for sequences without a checked position
+    int bad = ((status != nullptr && *status != 0) || (seq_flags != nullptr && seq_flags[b] != 0)) ? 1 : 0;
+    int cells = 0;
     double sum = 0.0;
     for (int s = threadIdx.x; s < n_check; s += kSeqThreads) {
         if (seq_of_slot[s] != b) continue;
@@ -576,7 +584,14 @@ __global__ void convert_states_kernel(const float* __restrict__ src, void* __res
     else reinterpret_cast<float*>(dst)[i] = src[i];
 }
 
-__global__ void load_states_kernel(const void* __restrict__ src, int dtype, size_t n, float* __restrict__ dst) {
+// Recorded states entering a segment come from another party.  A value that is not finite, or so large that
+// the first norm could overflow (|x| > kStateLimit), is replaced by zero and its sequence is marked in
+// seq_flags: such a sequence is rejected as a whole, and nothing non-finite reaches the packed buffers that
+// neighbouring sequences' attention tiles read.
+constexpr float kStateLimit = 1e15f;
+__global__ void load_states_kernel(const void* __restrict__ src, int dtype, size_t n, int d_model,
+                                   const int* __restrict__ seq_of_token, int* __restrict__ seq_flags,
+                                   float* __restrict__ dst) {
     const size_t i = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
     if (i >= n) return;  // n is a multiple of 4 (d_model % 64 == 0)
     float4 v;
@@ -586,7 +601,26 @@ __global__ void load_states_kernel(const void* __restrict__ src, int dtype, size
     } else {
         v = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(src) + i);
     }
+    const bool ok0 = fabsf(v.x) <= kStateLimit, ok1 = fabsf(v.y) <= kStateLimit;  // false for NaN
+    const bool ok2 = fabsf(v.z) <= kStateLimit, ok3 = fabsf(v.w) <= kStateLimit;
+    if (!(ok0 && ok1 && ok2 && ok3)) {
+        v.x = ok0 ? v.x : 0.f; v.y = ok1 ? v.y : 0.f; v.z = ok2 ? v.z : 0.f; v.w = ok3 ? v.w : 0.f;
+        if (seq_flags != nullptr) atomicOr(seq_flags + seq_of_token[i / static_cast<size_t>(d_model)], 1);
+    }
     *reinterpret_cast<float4*>(dst + i) = v;
+}
+
+// Exercise of the bounded wait every pipeline uses: one thread waits, with a short limit, on a barrier that
+// nothing will ever signal (no copy in flight, no tensor memory held), and returns with the timeout recorded.
+__global__ void wait_probe_kernel(long long limit_cycles, int* status, int* gave_up) {
+    __shared__ __align__(8) uint64_t bar_word;
+    if (threadIdx.x == 0) {
+        const uint32_t bar = smem_u32(&bar_word);
+        mbar_init(bar, 1);
+        fence_mbar_init();
+        const bool done = mbar_wait_limit(bar, 0u, status, limit_cycles);
+        if (gave_up) *gave_up = done ? 0 : 1;
+    }
 }
 
 __global__ void gather_tokens_kernel(const int* __restrict__ tokens, const int* __restrict__ src_index, int n,
@@ -644,18 +678,20 @@ cudaError_t launch_compare_rows(const float* hidden, const void* committed, int 
 }
 
 cudaError_t launch_verdict(const float* partials, int n_layers, int n_check, int n_tiles, int d, const TolDev& tol,
-                           const int* status, float* stats, uint8_t* pos_ok, int* first_bad_layer, cudaStream_t s) {
+                           const int* status, const int* seq_of_slot, const int* seq_flags, float* stats,
+                           uint8_t* pos_ok, int* first_bad_layer, cudaStream_t s) {
     if (n_check <= 0) return cudaSuccess;
-    verdict_kernel<<<(n_check + 3) / 4, 128, 0, s>>>(partials, n_layers, n_check, n_tiles, d, tol, status, stats,
-                                                      pos_ok, first_bad_layer);
+    verdict_kernel<<<(n_check + 3) / 4, 128, 0, s>>>(partials, n_layers, n_check, n_tiles, d, tol, status, seq_of_slot,
+                                                      seq_flags, stats, pos_ok, first_bad_layer);
     return cudaGetLastError();
 }
 
 cudaError_t launch_seq_verdict(const float* stats, const uint8_t* pos_ok, const int* seq_of_slot, int n_check,
-                               int n_layers, int batch, uint8_t* seq_ok, float* seq_score, cudaStream_t s) {
+                               int n_layers, int batch, const int* status, const int* seq_flags, uint8_t* seq_ok,
+                               float* seq_score, cudaStream_t s) {
     if (batch <= 0) return cudaSuccess;
-    seq_verdict_kernel<<<batch, kSeqThreads, 0, s>>>(stats, pos_ok, seq_of_slot, n_check, n_layers, batch, seq_ok,
-                                                        seq_score);
+    seq_verdict_kernel<<<batch, kSeqThreads, 0, s>>>(stats, pos_ok, seq_of_slot, n_check, n_layers, batch, status,
+                                                        seq_flags, seq_ok, seq_score);
     return cudaGetLastError();
 }
 
@@ -709,12 +745,17 @@ cudaError_t launch_decode_attention(const void* q, const void* kv_cache_layer, c
     if (rows <= 0) return cudaSuccess;
     const size_t smem = sizeof(float) * (static_cast<size_t>(head_dim) + static_cast<size_t>(max_keys));
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
-    static size_t configured = 48 * 1024;
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(decode_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(smem));
+    // the attribute belongs to the (function, device) pair: remember what each device was given
+    static size_t configured[64] = {0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (smem > 48 * 1024 && smem > configured[dev]) {
+        e = cudaFuncSetAttribute(decode_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        configured = smem;
+        configured[dev] = smem;
     }
     decode_attention_kernel<<<dim3(rows, n_heads), 128, smem, s>>>(
         reinterpret_cast<const __nv_bfloat16*>(q), reinterpret_cast<const __nv_bfloat16*>(kv_cache_layer), seq_start,
@@ -749,9 +790,16 @@ cudaError_t launch_convert_states(const float* src, void* dst, size_t n, int com
     return cudaGetLastError();
 }
 
-cudaError_t launch_load_states(const void* src, int dtype, size_t n, float* resid, cudaStream_t s) {
+cudaError_t launch_load_states(const void* src, int dtype, size_t n, int d_model, const int* seq_of_token,
+                               int* seq_flags, float* resid, cudaStream_t s) {
     if (n == 0) return cudaSuccess;
-    load_states_kernel<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, s>>>(src, dtype, n, resid);
+    load_states_kernel<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, s>>>(src, dtype, n, d_model, seq_of_token,
+                                                                                  seq_flags, resid);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_wait_probe(long long limit_cycles, int* status, int* gave_up, cudaStream_t s) {
+    wait_probe_kernel<<<1, 32, 0, s>>>(limit_cycles, status, gave_up);
     return cudaGetLastError();
 }
 

@@ -404,6 +404,9 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
+    // everything above touched only this CTA's own resources: it may run under the previous kernel's tail
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -641,6 +644,9 @@ gemm_bf16_tcgen05_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     cluster_wait();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
+    // everything above touched only the pair's own resources: it may run under the previous kernel's tail
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer (each CTA its own tiles)
@@ -801,13 +807,15 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
     cfg.blockDim = dim3(GEMM_THREADS);
     cfg.dynamicSmemBytes = P_GEMM_SMEM;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = p.overlap_prologue ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, gemm_bf16_tcgen05_pair<EPI>, ta, tb, q);
 }
 
@@ -822,8 +830,17 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmP
     const int num_tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
     if (num_tiles <= 0) return cudaSuccess;
     const int grid = num_tiles < num_sms ? num_tiles : num_sms;
-    gemm_bf16_tcgen05<EPI><<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tb, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = GEMM_SMEM;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.overlap_prologue ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, gemm_bf16_tcgen05<EPI>, ta, tb, p);
 }
 
 template <int EPI>

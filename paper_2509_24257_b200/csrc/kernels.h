@@ -59,6 +59,10 @@ struct GemmParams {
     // parts of the last, partly filled round of tiles; nullptr: no K split.  pairs_total is set by the launcher.
     int* split_flags;
     int pairs_total;
+    // 1: launch with programmatic stream serialisation, so that the kernel's prologue (barriers, tensor memory,
+    // descriptor prefetch) runs under the tail of the kernel before it in the stream; the kernel waits for that
+    // kernel's completion before it reads or writes any global memory.
+    int overlap_prologue;
     int* status;
 };
 
@@ -71,9 +75,10 @@ cudaError_t gemm_init();  // raises the dynamic shared memory limit of every ins
 
 // ------------------------------------------------------------------ attention
 // tmap_q / tmap_kv are 64-column boxes of 128 / 64 rows over the same [tokens][(H+2KV)dh] buffer.
+// overlap_prologue as in GemmParams; cu_seqlens_dev must not be written by the kernel just before in the stream.
 cudaError_t launch_attention_tc(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, const int* cu_seqlens_dev,
                                 int batch, int max_seqlen, int n_heads, int n_kv_heads, int head_dim, void* out,
-                                int* status, int num_sms, cudaStream_t stream);
+                                int* status, int num_sms, int overlap_prologue, cudaStream_t stream);
 cudaError_t attention_tc_init();
 
 // ------------------------------------------------------------------ small kernels
@@ -83,8 +88,10 @@ cudaError_t launch_slot_lists(const int* tok_of_slot, int n_check, int n_tokens,
                               cudaStream_t stream);
 cudaError_t launch_embed(const int* tokens, const void* table, int n_tokens, int d_model, int vocab, float* resid,
                          int* status, cudaStream_t stream);
-// resid[n] (fp32) = recorded states in `dtype` (VERILLM_BF16 / VERILLM_F32): input of a segment-local pass
-cudaError_t launch_load_states(const void* src, int dtype, size_t n, float* resid, cudaStream_t stream);
+// resid[n] (fp32) = recorded states in `dtype` (VERILLM_BF16 / VERILLM_F32): input of a segment-local pass.
+// Values that are not finite or beyond 1e15 in magnitude become 0 and mark their sequence in seq_flags[batch].
+cudaError_t launch_load_states(const void* src, int dtype, size_t n, int d_model, const int* seq_of_token,
+                               int* seq_flags, float* resid, cudaStream_t stream);
 cudaError_t launch_rmsnorm(const float* x, const void* gain, void* y, int rows, int d, float eps,
                            cudaStream_t stream);
 // The producer half of a folded norm as a kernel of its own (first layer of a pass, small batches):
@@ -98,11 +105,14 @@ struct TolDev {
     int bit_aware;
 };
 // partials: [n_layers][n_check][n_tiles][kNPart] -> stats [n_check][n_layers][NSTAT], pos_ok, first_bad_layer
+// seq_flags (optional, with seq_of_slot): sequences whose input was malformed; all their positions are rejected.
 cudaError_t launch_verdict(const float* partials, int n_layers, int n_check, int n_tiles, int d, const TolDev& tol,
-                           const int* status, float* stats, uint8_t* pos_ok, int* first_bad_layer,
-                           cudaStream_t stream);
+                           const int* status, const int* seq_of_slot, const int* seq_flags, float* stats,
+                           uint8_t* pos_ok, int* first_bad_layer, cudaStream_t stream);
+// status / seq_flags (both optional): a non-zero status word rejects every sequence, a flag its sequence.
 cudaError_t launch_seq_verdict(const float* stats, const uint8_t* pos_ok, const int* seq_of_slot, int n_check,
-                               int n_layers, int batch, uint8_t* seq_ok, float* seq_score, cudaStream_t stream);
+                               int n_layers, int batch, const int* status, const int* seq_flags, uint8_t* seq_ok,
+                               float* seq_score, cudaStream_t stream);
 
 // Threshold sensitivity: counts[v][4] += (honest accepted, honest rejected, attack accepted, attack rejected)
 // over the cells' reported statistics [n_cells][VERILLM_NSTAT] for each of n_variants tolerance sets.
@@ -142,6 +152,9 @@ cudaError_t launch_gather_rows(const float* resid, const int* row_of_slot, const
 cudaError_t launch_scatter_kv(const void* qkv, const int* dst_row, int rows, int n_heads, int n_kv_heads,
                               int head_dim, void* kv_cache_layer, cudaStream_t stream);
 cudaError_t launch_convert_states(const float* src, void* dst, size_t n, int commit_dtype, cudaStream_t stream);
+// One thread waits on a barrier nobody signals, for at most limit_cycles: *status receives
+// VERILLM_DEV_WAIT_TIMEOUT, *gave_up 1.
+cudaError_t launch_wait_probe(long long limit_cycles, int* status, int* gave_up, cudaStream_t stream);
 cudaError_t launch_gather_tokens(const int* tokens, const int* src_index, int n, int* out, cudaStream_t stream);
 
 }  // namespace vl

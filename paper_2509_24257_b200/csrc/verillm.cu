@@ -74,6 +74,10 @@ struct verillm_model {
     bf16 *xn = nullptr, *qkv = nullptr, *attn = nullptr, *mid = nullptr;
     int *pos_of_token = nullptr, *seq_of_token = nullptr, *slot_first = nullptr, *slot_next = nullptr;
     int *tok_of_slot = nullptr, *seq_of_slot = nullptr, *cu_dev = nullptr, *status = nullptr;
+    int* seq_flags = nullptr;  // [max_batch] sequences whose recorded input states were malformed
+    // Library-owned (pageable) copies of the caller's host arrays: an asynchronous copy out of pageable memory
+    // is staged before the call returns, so the caller's arrays, pinned or not, are free again at return.
+    std::vector<int> h_cu, h_tok_of_slot, h_seq_of_slot, h_claimed;
     float* partials = nullptr;
     int* split_flags = nullptr;  // K-part counters of the GEMMs' last round (one per pair of SMs)
     float* sumsq = nullptr;  // [max_tokens][n_tiles_d]: per-tile sums of squares of the residual rows (folded RMSNorm)
@@ -212,6 +216,7 @@ int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st
     p.status = status;
     p.M = r.M;
     p.pair = use_pair(r.M);
+    p.overlap_prologue = 1;  // the five kernels of a block chain their prologues under each other's tails
     // Tile walk in bands of 16 tile-rows for every projection (measured: bands of 4, 8, 32 and "all rows" are
     // no faster, also for the K = d_model projections whose activations would fit in L2).
     const int band_d = 16;
@@ -234,7 +239,7 @@ int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st
     CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, p.pair ? w.t_wqkv_h : w.t_wqkv, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_QKV, st);
     CU_TRY(launch_attention_tc(m->t_qkv_q, m->t_qkv_kv, r.cu_dev, r.batch, r.max_len, c.n_heads, c.n_kv_heads,
-                               c.head_dim, m->attn, status, m->num_sms, st));
+                               c.head_dim, m->attn, status, m->num_sms, 1, st));
     prof_mark(m, VERILLM_PROF_ATTENTION, st);
     p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
     p.group_m = band_d;
@@ -331,6 +336,7 @@ void verillm_free(verillm_model* m) {
     cudaFree(m->resid); cudaFree(m->xn); cudaFree(m->qkv); cudaFree(m->attn); cudaFree(m->mid);
     cudaFree(m->pos_of_token); cudaFree(m->seq_of_token); cudaFree(m->slot_first); cudaFree(m->slot_next);
     cudaFree(m->tok_of_slot); cudaFree(m->seq_of_slot); cudaFree(m->cu_dev); cudaFree(m->status);
+    cudaFree(m->seq_flags);
     cudaFree(m->partials); cudaFree(m->sumsq); cudaFree(m->split_flags); cudaFree(m->rope_cs);
     cudaFree(m->lm_head); cudaFree(m->tm_y); cudaFree(m->tm_rec); cudaFree(m->tm_claimed);
     DecodeState& d = m->dec;
@@ -456,6 +462,7 @@ int verillm_load_weights(const verillm_config* cfg, const verillm_weights* weigh
     TRY_RC(dev_alloc(&m->seq_of_slot, NC));
     TRY_RC(dev_alloc(&m->cu_dev, static_cast<size_t>(c.max_batch) + 1));
     TRY_RC(dev_alloc(&m->status, 1));
+    TRY_RC(dev_alloc(&m->seq_flags, static_cast<size_t>(c.max_batch)));
     TRY_RC(dev_alloc(&m->partials, static_cast<size_t>(c.n_layers) * NC * m->n_tiles_d * kNPart));
     TRY_RC(dev_alloc(&m->sumsq, T * m->n_tiles_d));
     TRY_RC(dev_alloc(&m->split_flags, 256));
@@ -535,8 +542,9 @@ static int verify_impl(verillm_model* m, const int32_t* tokens, const void* stat
     if (n_check > 0 && (!committed_hidden || !rep->stats || !rep->pos_ok || !rep->first_bad_layer)) return VERILLM_E_INVAL;
     int M = 0, max_len = 0, rc;
     if ((rc = check_batch(m, cu_seqlens, batch, &M, &max_len))) return rc;
-    std::vector<int> tok_of_slot;
-    if ((rc = check_slots(m, cu_seqlens, batch, check_seq, check_pos, n_check, &tok_of_slot))) return rc;
+    if ((rc = check_slots(m, cu_seqlens, batch, check_seq, check_pos, n_check, &m->h_tok_of_slot))) return rc;
+    m->h_cu.assign(cu_seqlens, cu_seqlens + batch + 1);
+    m->h_seq_of_slot.assign(check_seq, check_seq + n_check);
 
     const verillm_config& c = m->cfg;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -544,17 +552,29 @@ static int verify_impl(verillm_model* m, const int32_t* tokens, const void* stat
     m->prof.n = 0;
     prof_mark(m, -1, st);
     CU_TRY(cudaMemsetAsync(rep->status, 0, sizeof(int), st));
-    CU_TRY(cudaMemcpyAsync(m->cu_dev, cu_seqlens, sizeof(int) * (batch + 1), cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(m->cu_dev, m->h_cu.data(), sizeof(int) * (batch + 1), cudaMemcpyHostToDevice, st));
     if (n_check > 0) {
-        CU_TRY(cudaMemcpyAsync(m->tok_of_slot, tok_of_slot.data(), sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
-        CU_TRY(cudaMemcpyAsync(m->seq_of_slot, check_seq, sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(m->tok_of_slot, m->h_tok_of_slot.data(), sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(m->seq_of_slot, m->h_seq_of_slot.data(), sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+    }
+    // Key/value tiles of the last sequence reach up to 63 rows past the last token; those rows still hold
+    // what an earlier, larger call left there.  Their probabilities are zero, but zero times a non-finite
+    // value is not: clear them.
+    {
+        const size_t tail = std::min<size_t>(static_cast<size_t>(c.max_tokens) - M, 128);
+        if (tail > 0) CU_TRY(cudaMemsetAsync(m->qkv + static_cast<size_t>(M) * m->n_qkv, 0, tail * m->n_qkv * sizeof(bf16), st));
     }
     CU_TRY(launch_token_maps(m->cu_dev, batch, M, m->pos_of_token, m->seq_of_token, st));
     CU_TRY(launch_slot_lists(m->tok_of_slot, n_check, M, m->slot_first, m->slot_next, st));
-    if (tokens)
+    int* seq_flags = nullptr;
+    if (tokens) {
         CU_TRY(launch_embed(tokens, m->embed, M, c.d_model, c.vocab, m->resid, rep->status, st));
-    else
-        CU_TRY(launch_load_states(states_in, in_dtype, static_cast<size_t>(M) * c.d_model, m->resid, st));
+    } else {
+        seq_flags = m->seq_flags;
+        CU_TRY(cudaMemsetAsync(seq_flags, 0, sizeof(int) * batch, st));
+        CU_TRY(launch_load_states(states_in, in_dtype, static_cast<size_t>(M) * c.d_model, c.d_model, m->seq_of_token,
+                                  seq_flags, m->resid, st));
+    }
     launches += 2 + (n_check > 0 ? 1 : 0);
     prof_mark(m, VERILLM_PROF_SETUP, st);
 
@@ -573,9 +593,9 @@ static int verify_impl(verillm_model* m, const int32_t* tokens, const void* stat
         if ((rc = run_layer(m, l, run, rep->status, st, &launches))) return rc;
     }
     CU_TRY(launch_verdict(m->partials, l1 - l0, n_check, m->n_tiles_d, c.d_model, tol_dev(*tol), rep->status,
-                          rep->stats, rep->pos_ok, rep->first_bad_layer, st));
-    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, m->seq_of_slot, n_check, l1 - l0, batch, rep->seq_ok,
-                              rep->seq_score, st));
+                          m->seq_of_slot, seq_flags, rep->stats, rep->pos_ok, rep->first_bad_layer, st));
+    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, m->seq_of_slot, n_check, l1 - l0, batch, rep->status, seq_flags,
+                              rep->seq_ok, rep->seq_score, st));
     launches += (n_check > 0 ? 1 : 0) + 1;
     prof_mark(m, VERILLM_PROF_VERDICT, st);
     m->last_launches = launches;
@@ -620,11 +640,14 @@ int verillm_compare(const float* hidden, const void* committed, int32_t commit_d
     CU_TRY(cudaMallocAsync(reinterpret_cast<void**>(&partials), rows * kNPart * sizeof(float), st));
     CU_TRY(cudaMallocAsync(reinterpret_cast<void**>(&seq_dev), sizeof(int) * n_check, st));
     CU_TRY(cudaMemsetAsync(rep->status, 0, sizeof(int), st));
-    CU_TRY(cudaMemcpyAsync(seq_dev, check_seq, sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+    // (a library-owned pageable copy is staged before the call returns, whatever memory the caller's array is in)
+    const std::vector<int> seq_host(check_seq, check_seq + n_check);
+    CU_TRY(cudaMemcpyAsync(seq_dev, seq_host.data(), sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
     CU_TRY(launch_compare_rows(hidden, committed, static_cast<int>(rows), d_model, cmp_params(*tol, commit_dtype), partials, st));
-    CU_TRY(launch_verdict(partials, n_layers, n_check, 1, d_model, tol_dev(*tol), rep->status, rep->stats, rep->pos_ok,
-                          rep->first_bad_layer, st));
-    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, seq_dev, n_check, n_layers, batch, rep->seq_ok, rep->seq_score, st));
+    CU_TRY(launch_verdict(partials, n_layers, n_check, 1, d_model, tol_dev(*tol), rep->status, nullptr, nullptr,
+                          rep->stats, rep->pos_ok, rep->first_bad_layer, st));
+    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, seq_dev, n_check, n_layers, batch, rep->status, nullptr,
+                              rep->seq_ok, rep->seq_score, st));
     CU_TRY(cudaFreeAsync(partials, st));
     CU_TRY(cudaFreeAsync(seq_dev, st));
     return VERILLM_OK;
@@ -642,6 +665,9 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 // Device address of the array on each device, resolved on the first call made with that device current.
 // (In host code `g_noalloc_scratch` is only a handle for the runtime, never a pointer a kernel may use.)
 static void* g_noalloc_ptr[64] = {nullptr};
+// Pageable host copy of the caller's check_seq (copies out of pageable memory are staged before the copy call
+// returns, so the caller's array is free again at return even if it is pinned).  Shared like the device array.
+static int g_noalloc_host_seq[kNoAllocMaxChecks];
 
 int verillm_compare_noalloc(const float* hidden, const void* committed, int32_t commit_dtype, int32_t n_layers,
                             int32_t n_check, int32_t d_model, const int32_t* check_seq, int32_t batch,
@@ -672,11 +698,13 @@ int verillm_compare_noalloc(const float* hidden, const void* committed, int32_t 
     // the array still holds the previous call's records: wipe the part this call will read
     CU_TRY(cudaMemsetAsync(partials, 0, rows * kNPart * sizeof(float), st));
     CU_TRY(cudaMemsetAsync(rep->status, 0, sizeof(int), st));
-    CU_TRY(cudaMemcpyAsync(seq_dev, check_seq, sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+    std::memcpy(g_noalloc_host_seq, check_seq, sizeof(int) * n_check);
+    CU_TRY(cudaMemcpyAsync(seq_dev, g_noalloc_host_seq, sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
     CU_TRY(launch_compare_rows(hidden, committed, static_cast<int>(rows), d_model, cmp_params(*tol, commit_dtype), partials, st));
-    CU_TRY(launch_verdict(partials, n_layers, n_check, 1, d_model, tol_dev(*tol), rep->status, rep->stats, rep->pos_ok,
-                          rep->first_bad_layer, st));
-    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, seq_dev, n_check, n_layers, batch, rep->seq_ok, rep->seq_score, st));
+    CU_TRY(launch_verdict(partials, n_layers, n_check, 1, d_model, tol_dev(*tol), rep->status, nullptr, nullptr,
+                          rep->stats, rep->pos_ok, rep->first_bad_layer, st));
+    CU_TRY(launch_seq_verdict(rep->stats, rep->pos_ok, seq_dev, n_check, n_layers, batch, rep->status, nullptr,
+                              rep->seq_ok, rep->seq_score, st));
     return VERILLM_OK;
 }
 
@@ -710,7 +738,8 @@ int verillm_token_match(verillm_model* m, const float* last_hidden, const int32_
     if (n_check > m->cfg.max_checks) return VERILLM_E_SHAPE;
     const verillm_config& c = m->cfg;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-    CU_TRY(cudaMemcpyAsync(m->tm_claimed, claimed, sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
+    m->h_claimed.assign(claimed, claimed + n_check);
+    CU_TRY(cudaMemcpyAsync(m->tm_claimed, m->h_claimed.data(), sizeof(int) * n_check, cudaMemcpyHostToDevice, st));
     CU_TRY(launch_rmsnorm(last_hidden, m->final_norm, m->tm_y, n_check, c.d_model, c.rms_eps, st));
     GemmParams p;
     std::memset(&p, 0, sizeof(p));
@@ -736,9 +765,12 @@ int verillm_spot_check(const float* hidden, int32_t n_rows, int32_t d_model, con
     int* rows = reinterpret_cast<int*>(buf);
     int* cols = rows + n;
     float* ref = reinterpret_cast<float*>(cols + n);
-    CU_TRY(cudaMemcpyAsync(rows, sample_row, n * 4, cudaMemcpyHostToDevice, st));
-    CU_TRY(cudaMemcpyAsync(cols, sample_col, n * 4, cudaMemcpyHostToDevice, st));
-    CU_TRY(cudaMemcpyAsync(ref, reference, n * 4, cudaMemcpyHostToDevice, st));
+    // one library-owned pageable copy of the three arrays: staged before the copy call returns
+    std::vector<int> host(3 * n);
+    std::memcpy(host.data(), sample_row, n * 4);
+    std::memcpy(host.data() + n, sample_col, n * 4);
+    std::memcpy(host.data() + 2 * n, reference, n * 4);
+    CU_TRY(cudaMemcpyAsync(buf, host.data(), n * 12, cudaMemcpyHostToDevice, st));
     CU_TRY(launch_spot_check(hidden, d_model, rows, cols, ref, n_samples, eps, theta, agree_out, p_hat_out, verdict_out, st));
     CU_TRY(cudaFreeAsync(buf, st));
     return VERILLM_OK;
@@ -918,6 +950,16 @@ int verillm_decode_commit(verillm_model* m, const int32_t* tokens, const int32_t
     return VERILLM_OK;
 }
 
+int verillm_selftest_wait_timeout(int64_t limit_cycles, int32_t* status, int32_t* gave_up, void* cuda_stream) {
+    if (!status || limit_cycles < 1 || limit_cycles > 2000000000LL) return VERILLM_E_INVAL;
+    int rc = ensure_init();
+    if (rc) return rc;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    CU_TRY(cudaMemsetAsync(status, 0, sizeof(int), st));
+    CU_TRY(launch_wait_probe(limit_cycles, status, gave_up, st));
+    return VERILLM_OK;
+}
+
 int verillm_op_gemm(const void* a, const void* b, void* cmat, int32_t M, int32_t N, int32_t K, int32_t out_f32,
                     int32_t* status, void* cuda_stream) {
     if (!a || !b || !cmat || M < 1 || N < 1 || K < 1) return VERILLM_E_INVAL;
@@ -961,7 +1003,7 @@ int verillm_op_attention(const void* qkv, const int32_t* cu_seqlens, int32_t bat
     CU_TRY(cudaGetDevice(&dev));
     CU_TRY(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
     CU_TRY(launch_attention_tc(tq, tkv, cu_seqlens, batch, max_seqlen, n_heads, n_kv_heads, head_dim, out, nullptr,
-                               num_sms, reinterpret_cast<cudaStream_t>(cuda_stream)));
+                               num_sms, 0, reinterpret_cast<cudaStream_t>(cuda_stream)));
     return VERILLM_OK;
 }
 

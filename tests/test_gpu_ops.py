@@ -213,3 +213,84 @@ def test_merkle_roots_are_bit_exact(n_vec, d):
     with pytest.raises(vb.VerillmError) as e:
         vb.merkle_roots(torch.zeros(1, 12801, device=DEV))
     assert e.value.code == vb.E_SHAPE
+
+
+def _exact_rows(L, n, d, seed):
+    """Committed rows and deviations whose statistics are exact in float32: every value is a small multiple of
+    2^-10, most deviations are zero, a few are +-2^-18 (below the 1e-5 of Q_small) or multiples of 1/8."""
+    rng = np.random.default_rng(seed)
+    c = rng.integers(-2048, 2048, (L, n, d)) / 1024.0
+    delta = np.zeros((L, n, d))
+    for l in range(L):
+        for i in range(n):
+            k = rng.integers(0, d // 2 + 1)
+            idx = rng.choice(d, k, replace=False)
+            delta[l, i, idx] = rng.choice([2.0 ** -18, -2.0 ** -18, 0.125, -0.125, 0.25, 0.5, -0.75], k)
+    return (c + delta).astype(np.float32), c.astype(np.float32)
+
+
+def test_every_float_test_of_the_verdict_matches_oracle_bit_for_bit():
+    """max |Delta|, MAE, Z_large and Q_small enabled in the standalone comparison and in the threshold sweep, on
+    rows whose statistics are exact in float32, with each threshold set to a value some row attains exactly:
+    verdicts, first failing layers and sweep counts equal the oracle's."""
+    L, n, d = 3, 40, 64
+    hidden, comm = _exact_rows(L, n, d, 77)
+    check_seq = (np.arange(n) % 3).astype(np.int32)
+    base = dict(rel_l2=0.0, tau_large=0.125)
+    stats_o = np.transpose(vo.compare_stats(hidden.astype(np.float64), comm.astype(np.float64), "f32", vo.Tol(**base)), (1, 0, 2))
+    med = lambda name: float(np.median(stats_o[..., vo.STAT_NAMES.index(name)]))
+    variants = [
+        dict(max_abs=0.5), dict(mae=med("mae")), dict(z_large_max=med("z_large")), dict(q_small_min=med("q_small")),
+        dict(z_large_max=0.0), dict(q_small_min=1.0),
+        dict(max_abs=0.5, mae=med("mae"), z_large_max=med("z_large"), q_small_min=med("q_small")),
+    ]
+    hid_t, com_t = torch.from_numpy(hidden).to(DEV), torch.from_numpy(comm).to(DEV)
+    seen = set()
+    for kw in variants:
+        tol_o, tol_g = vo.Tol(**base, **kw), vb.default_tol(**base, **kw)
+        rep = vb.compare(hid_t, com_t, check_seq, 3, tol_g).cpu()
+        for j, nm in enumerate(vo.STAT_NAMES):
+            if nm not in ("rel_l2", "l2_delta", "l2_ref"):  # everything but the square roots is exact here:
+                # sums and counts exactly, ratios of counts (P_w, P_m) as the correctly rounded float32 quotient
+                assert np.array_equal(rep["stats"][..., j].astype(np.float32), stats_o[..., j].astype(np.float32)), nm
+        pos_ok, first_bad, seq_ok, _ = vo.verdict(stats_o, check_seq, 3, tol_o)
+        assert np.array_equal(rep["pos_ok"], pos_ok) and np.array_equal(rep["first_bad_layer"], first_bad), kw
+        assert np.array_equal(rep["seq_ok"], seq_ok), kw
+        seen.add((int(pos_ok.sum()) > 0, int(pos_ok.sum()) < n))
+    assert (True, True) in seen  # thresholds that split the rows, not all-or-nothing
+    # the same tests applied afterwards to the reported statistics
+    rep = vb.compare(hid_t, com_t, check_seq, 3, vb.default_tol(**base))
+    cells = rep.stats[:n].reshape(-1, vb.NSTAT).contiguous()
+    attack = torch.from_numpy((np.arange(n * L) % 2).astype(np.uint8)).to(DEV)
+    counts = vb.threshold_sweep(cells, attack, [vb.default_tol(**base, **kw) for kw in variants]).cpu().numpy()
+    counts_o = vo.threshold_sweep(cells.cpu().numpy(), attack.cpu().numpy(), [vo.Tol(**base, **kw) for kw in variants])
+    assert np.array_equal(counts, counts_o)
+    assert (counts[:4, 0] > 0).all() and (counts[:4, 1] > 0).all()
+
+
+def test_relaxed_value_test_on_a_full_row_equals_the_spot_check():
+    """Position-granular form of the relaxed on-chain test: tau_large = eps, z_large_max = 1 - theta on a whole
+    row decides like the sampled-scalar spot check over all d entries of that row, on the GPU and in the oracle."""
+    rng = np.random.default_rng(13)
+    n, d, eps = 24, 256, 0.125
+    comm = (rng.integers(-4096, 4096, (1, n, d)) / 1024.0).astype(np.float32)
+    hidden = comm.copy()
+    for i in range(n):
+        far = rng.choice(d, int(rng.integers(0, d // 2)), replace=False)
+        hidden[0, i, far] += rng.choice([-0.5, 0.25, 1.0], len(far)).astype(np.float32)
+        hidden[0, i, (far + 1) % d] += np.float32(0.125)  # exactly eps: agrees
+    hidden[0, 0] = comm[0, 0]
+    hidden[0, 1, : d // 4] = comm[0, 1, : d // 4] + 1.0  # p_hat = 0.75 exactly (the rest of row 1 is reset below)
+    hidden[0, 1, d // 4:] = comm[0, 1, d // 4:]
+    hid_t, com_t = torch.from_numpy(hidden).to(DEV), torch.from_numpy(comm).to(DEV)
+    cols = np.arange(d)
+    for theta in (0.5, 0.75, 1.0):
+        kw = dict(rel_l2=0.0, tau_large=eps, z_large_max=1.0 - theta)
+        rep = vb.compare(hid_t, com_t, np.zeros(n, np.int32), 1, vb.default_tol(**kw)).cpu()
+        stats_o = vo.compare_stats(hidden[0].astype(np.float64), comm[0].astype(np.float64), "f32", vo.Tol(**kw))
+        for i in range(n):
+            _, p_hat, ok = vb.spot_check(hid_t[0], np.full(d, i), cols, comm[0, i], eps, theta)
+            _, p_hat_o, ok_o = vo.spot_check(hidden[0], np.full(d, i), cols, comm[0, i], eps, theta)
+            assert float(p_hat.item()) == p_hat_o and bool(ok.item()) == ok_o
+            assert bool(rep["pos_ok"][i]) == ok_o == bool(vo.layer_passes(stats_o[i], vo.Tol(**kw))), (theta, i)
+    assert rep["pos_ok"][0] == 1

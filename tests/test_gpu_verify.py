@@ -332,3 +332,122 @@ def test_segment_local_verification_matches_oracle(small):
     with pytest.raises(vb.VerillmError) as e:
         model.verify_segment(states, 3, 3, synth.cu_seqlens(wl), comm_t.to(DEV), cs, cp)
     assert e.value.code == vb.E_RANGE
+
+
+def test_nonfinite_recorded_states_reject_only_their_sequence(tiny):
+    """Two packed sequences whose lengths are not multiples of the 64-key tile: the last key tile of the first
+    covers the first rows of the second.  Inf / NaN (and an absurdly large value) in the second sequence's
+    recorded input states reject that sequence as a whole, as the exact recomputation does (one such entry
+    makes every state of its sequence non-finite), while the first sequence's statistics and verdict are those
+    of the clean run, bit for bit; a following, smaller clean call on the same handle is unaffected."""
+    wl, _, om, _, _, _, _ = tiny
+    rng = np.random.default_rng(21)
+    lens = [37, 45]
+    states = [vo.round_to_bf16(rng.standard_normal((n, wl.shape.d_model)) * 0.5) for n in lens]
+    cu = np.array([0, 37, 82], np.int32)
+    cs = np.array([0, 0, 1, 1, 0], np.int32)
+    cp = np.array([36, 3, 0, 44, 20], np.int32)
+    outs = vo.forward_segment_batch(om, states, 0, 1)
+    honest = np.stack([outs[s][:, p] for s, p in zip(cs, cp)], axis=1)
+    comm = synth.to_commit_dtype(honest, "bf16").to(DEV)
+    model = vb.Model(wl.shape, 128, len(cs), 2, DEV)
+    model.load_globals(synth.embed_weights(wl, DEV), synth.final_norm_weights(wl, DEV))
+    model.load_layer(0, synth.layer_weights(wl, 0, DEV))
+    clean_in = synth.to_commit_dtype(np.concatenate(states), "f32")
+    clean = model.verify_segment(clean_in.to(DEV), 0, 1, cu, comm, cs, cp, want_hidden=True).cpu()
+    assert clean["pos_ok"].all() and clean["seq_ok"].tolist() == [1, 1]
+    for bad_value, where in ((float("inf"), (37 + 5, 7)), (float("nan"), (37 + 44, 255)), (-3e20, (37 + 0, 0))):
+        bad_in = clean_in.clone()
+        bad_in[where] = bad_value
+        g = model.verify_segment(bad_in.to(DEV), 0, 1, cu, comm, cs, cp, want_hidden=True).cpu()
+        assert g["status"] == 0
+        assert g["seq_ok"].tolist() == [1, 0]
+        assert g["pos_ok"].tolist() == [1, 1, 0, 0, 1] and g["first_bad_layer"].tolist() == [-1, -1, 0, 0, -1]
+        first = [0, 1, 4]
+        assert np.array_equal(g["stats"][first], clean["stats"][first])
+        assert np.array_equal(g["hidden"][:, first], clean["hidden"][:, first])
+        assert np.isfinite(g["hidden"]).all()
+        assert g["seq_score"][0] == clean["seq_score"][0]
+        # the oracle on the same input: every state of the poisoned sequence is non-finite, the other is untouched
+        bad_states = [states[0], bad_in[37:].to(torch.float64).numpy()]
+        with np.errstate(all="ignore"):
+            o = vo.verify_segment(om, bad_states, 0, 1, comm.cpu().to(torch.float64).numpy(), cs, cp, vo.Tol(), "bf16")
+        if abs(bad_value) > 1e30 or bad_value != bad_value:
+            assert np.array_equal(g["pos_ok"], o.pos_ok) and np.array_equal(g["seq_ok"], o.seq_ok)
+            assert np.array_equal(g["first_bad_layer"], o.first_bad_layer)
+        # a smaller clean call afterwards (the first sequence alone) reproduces the clean result
+        sub = model.verify_segment(clean_in[:37].to(DEV), 0, 1, cu[:2], comm[:, first].contiguous(), cs[first], cp[first],
+                                   want_hidden=True).cpu()
+        assert np.array_equal(sub["stats"], clean["stats"][first]) and sub["seq_ok"].tolist() == [1]
+    model.close()
+
+
+def test_device_error_rejects_sequences_without_checked_positions(tiny):
+    """An out-of-vocabulary token invalidates the whole call: also a sequence that has no checked position, and a
+    call without any check, must come back rejected."""
+    wl, tokens, om, cs, cp, committed, model = tiny
+    small = vb.Model(wl.shape, 64, 4, 2, DEV)
+    small.load_globals(synth.embed_weights(wl, DEV), synth.final_norm_weights(wl, DEV))
+    small.load_layer(0, synth.layer_weights(wl, 0, DEV))
+    toks = torch.from_numpy(tokens.reshape(-1)[:64].copy()).to(DEV)
+    cu = np.array([0, 40, 64], np.int32)
+    comm = synth.to_commit_dtype(committed[:, :2], "bf16").to(DEV)
+    ok = small.verify_prefill(toks, cu, comm, [0, 0], [int(cp[0]) % 40, int(cp[1]) % 40]).cpu()
+    assert ok["status"] == 0 and ok["seq_ok"][1] == 1  # sequence 1 has no checked position
+    bad = toks.clone()
+    bad[50] = -7  # inside sequence 1
+    rep = small.verify_prefill(bad, cu, comm, [0, 0], [int(cp[0]) % 40, int(cp[1]) % 40]).cpu()
+    assert rep["status"] == vb.DEV_TOKEN_RANGE and rep["seq_ok"].tolist() == [0, 0] and not rep["pos_ok"].any()
+    rep = small.verify_prefill(bad, cu, None, [], []).cpu()
+    assert rep["status"] == vb.DEV_TOKEN_RANGE and rep["seq_ok"].tolist() == [0, 0]
+    small.close()
+
+
+def test_pinned_host_arrays_may_be_overwritten_when_the_call_returns(tiny):
+    """The header's promise: host arrays are free again at return.  With page-locked arrays a direct asynchronous
+    copy would still be queued behind the work already on the stream; the library copies them first."""
+    wl, tokens, om, cs, cp, committed, model = tiny
+    comm = synth.to_commit_dtype(committed, "bf16").to(DEV)
+    flat = torch.from_numpy(tokens.reshape(-1)).to(DEV)
+    ref = model.verify_prefill(flat, synth.cu_seqlens(wl), comm, cs, cp, want_hidden=True).cpu()
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).pin_memory()
+    cu_p, cs_p, cp_p = pin(synth.cu_seqlens(wl)), pin(cs), pin(cp)
+    # keep the stream busy so that the call's own copies cannot have run when it returns
+    a = torch.randn(4096, 4096, device=DEV)
+    for _ in range(20):
+        a = a @ a * 1e-2
+    rep = model.verify_prefill(flat, cu_p.numpy(), comm, cs_p.numpy(), cp_p.numpy(), want_hidden=True)
+    cu_p.fill_(0); cs_p.fill_(0); cp_p.fill_(63)  # the caller reuses its arrays at once
+    torch.cuda.synchronize()
+    g = rep.cpu()
+    assert np.array_equal(g["stats"], ref["stats"]) and np.array_equal(g["hidden"], ref["hidden"])
+    assert np.array_equal(g["seq_ok"], ref["seq_ok"]) and np.array_equal(g["seq_score"], ref["seq_score"])
+    # the standalone comparison keeps the same promise for its slot-to-sequence map
+    hid = torch.from_numpy(ref["hidden"]).to(DEV)
+    seq_of = (np.arange(len(cs)) % 2).astype(np.int32)
+    ref2 = vb.compare(hid, comm, seq_of, 2).cpu()
+    seq_p = pin(seq_of)
+    for _ in range(20):
+        a = a @ a * 1e-2
+    r2 = vb.compare(hid, comm, seq_p.numpy(), 2)
+    seq_p.fill_(1)  # every slot would move to sequence 1
+    torch.cuda.synchronize()
+    r2 = r2.cpu()
+    assert np.array_equal(r2["stats"], ref2["stats"]) and np.array_equal(r2["seq_score"], ref2["seq_score"])
+    assert ref2["seq_score"][0] != ref2["seq_score"][1]
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable(tiny):
+    """Failure detection: the wait every pipeline uses, given a short limit and a barrier nothing signals, gives
+    up, records VERILLM_DEV_WAIT_TIMEOUT and returns; the next verification on the same context is correct."""
+    wl, tokens, om, cs, cp, committed, model = tiny
+    status, gave_up = vb.selftest_wait_timeout(200_000, DEV)  # about 0.1 ms of SM clocks
+    torch.cuda.synchronize()
+    assert int(status.item()) == vb.DEV_WAIT_TIMEOUT and int(gave_up.item()) == 1
+    with pytest.raises(vb.VerillmError):
+        vb.selftest_wait_timeout(0, DEV)
+    with pytest.raises(vb.VerillmError):
+        vb.selftest_wait_timeout(10 ** 12, DEV)  # limits beyond a second or so are refused
+    g, o = run_both(model, om, wl, tokens, committed, cs, cp)
+    assert_parity(g, o)
+    assert g["pos_ok"].all()

@@ -559,3 +559,115 @@ def test_fake_quantise_grid_and_error_bound():
         assert torch.allclose(k, torch.round(k), atol=1e-4) and float(k.abs().max()) <= qmax + 1e-4
         assert float(((q - w).abs() / step).max()) <= 0.5 + 1e-5
         assert torch.allclose(q.abs().amax(dim=1), w.abs().amax(dim=1))
+
+
+# ----------------------------------------------------------------------------- every branch of the verdict
+
+
+def _worked_row():
+    """Eight deviations whose statistics are exact binary fractions: 0.5, -0.25, 2^-18 and 0.125 beside four
+    zeros.  MAE = (0.875 + 2^-18) / 8, Q_small = 5/8 (the zeros and 2^-18 <= 1e-5), Z_large at tau = 0.125 is
+    2/8 (0.125 itself is not above tau), max |Delta| = 0.5."""
+    c = np.array([1.0, -2.0, 0.5, 0.0, 3.0, -1.0, 0.25, 1.5])
+    delta = np.array([0.5, -0.25, 0.0, 0.0, 0.0, 0.0, 2.0 ** -18, 0.125])
+    return c + delta, c
+
+
+def test_each_float_test_of_the_verdict_at_and_past_its_threshold():
+    """Offline battery T_off (MAE, Z_large, Q_small) and max |Delta|, one test enabled at a time: the value exactly
+    at the threshold accepts (b = 1[T_v <= tau]), the next representable threshold on the wrong side rejects,
+    and the documented "off" values switch the test off."""
+    h, c = _worked_row()
+    base = dict(rel_l2=0.0, tau_large=0.125)
+    s = vo.compare_stats(h, c, "f32", vo.Tol(**base))
+    v = dict(zip(vo.STAT_NAMES, s))
+    mae = 0.109375 + 2.0 ** -21
+    assert v["mae"] == mae and v["q_small"] == 0.625 and v["z_large"] == 0.25 and v["max_abs"] == 0.5
+    ok = lambda **kw: bool(vo.layer_passes(s, vo.Tol(**{**base, **kw})))
+    assert ok()  # nothing enabled: accept
+    # MAE <= tau
+    assert ok(mae=mae) and ok(mae=1.0) and not ok(mae=np.nextafter(mae, 0.0)) and not ok(mae=0.05)
+    assert ok(mae=0.0) and ok(mae=-1.0)  # <= 0 disables
+    # max |Delta| <= tau
+    assert ok(max_abs=0.5) and not ok(max_abs=np.nextafter(0.5, 0.0)) and ok(max_abs=0.0) and ok(max_abs=-3.0)
+    # Z_large <= z_large_max (a fraction of large deviations that is too high rejects)
+    assert ok(z_large_max=0.25) and ok(z_large_max=0.9) and not ok(z_large_max=np.nextafter(0.25, 0.0))
+    assert not ok(z_large_max=0.0)  # zero is an enabled threshold: no large deviation allowed at all
+    assert ok(z_large_max=-1.0) and ok(z_large_max=-1e-9)  # negative disables
+    # Q_small >= q_small_min (too few tiny deviations rejects)
+    assert ok(q_small_min=0.625) and ok(q_small_min=0.1) and not ok(q_small_min=np.nextafter(0.625, 1.0))
+    assert not ok(q_small_min=1.0)
+    assert ok(q_small_min=0.0) and ok(q_small_min=-0.5)  # <= 0 disables
+    # an identical pair passes every enabled test at its strictest setting
+    z = vo.compare_stats(c, c, "f32", vo.Tol(**base))
+    assert vo.layer_passes(z, vo.Tol(rel_l2=1e-30, max_abs=1e-30, mae=1e-30, tau_large=0.0, z_large_max=0.0, q_small_min=1.0))
+    # the tests combine by AND: one failing test rejects whatever the others say
+    assert ok(mae=1.0, max_abs=1.0, z_large_max=1.0, q_small_min=0.5)
+    assert not ok(mae=1.0, max_abs=1.0, z_large_max=1.0, q_small_min=0.7)
+    assert not ok(mae=1.0, max_abs=0.4, z_large_max=1.0, q_small_min=0.5)
+
+
+def test_relaxed_value_test_is_the_z_large_test_on_a_full_row():
+    """The relaxed on-chain test (|v_j - V_j| <= eps on sampled entries, agreement rate p_hat >= theta) applied to
+    every entry of a row decides like Z_large with tau_large = eps and z_large_max = 1 - theta: Z_large is the
+    fraction above eps, p_hat the fraction at or below it."""
+    rng = np.random.default_rng(11)
+    d, eps = 64, 0.125
+    cols = np.arange(d)
+    for n_far in (0, 5, 16, 17, 40, 64):
+        c = rng.standard_normal(d)
+        delta = rng.uniform(-0.1, 0.1, d)
+        far = rng.choice(d, n_far, replace=False)
+        delta[far] = rng.choice([-1.0, 1.0], n_far) * rng.uniform(0.2, 0.9, n_far)
+        if n_far:
+            delta[far[0]] = 0.125 if n_far == 64 else 0.5  # exactly eps agrees (<=), it is not "large" (>)
+        h = (c + delta).astype(np.float32).astype(np.float64)
+        c = c.astype(np.float32).astype(np.float64)
+        agree, p_hat, _ = vo.spot_check(h[None, :], np.zeros(d, int), cols, c, eps, 0.5)
+        for theta in (0.25, 0.5, 0.75, 0.9, 1.0):  # 1 - theta is exact for these in binary except 0.9
+            tol = vo.Tol(rel_l2=0.0, tau_large=eps, z_large_max=1.0 - theta)
+            s = vo.compare_stats(h, c, "f32", tol)
+            z = s[vo.STAT_NAMES.index("z_large")]
+            assert z == 1.0 - agree.sum() / d
+            on_chain = vo.spot_check(h[None, :], np.zeros(d, int), cols, c, eps, theta)[2]
+            if abs((1.0 - z) - theta) > 1e-6:  # away from the rounding of 1 - 0.9
+                assert bool(vo.layer_passes(s, tol)) == on_chain, (n_far, theta)
+    # the boundary itself with exact fractions: 16 of 64 far -> p_hat = 0.75 = theta accepts, 17 rejects
+    for n_far, expect in ((16, True), (17, False)):
+        c = np.zeros(d)
+        h = np.where(np.arange(d) < n_far, 1.0, 0.0)
+        tol = vo.Tol(rel_l2=0.0, tau_large=eps, z_large_max=0.25)
+        assert bool(vo.layer_passes(vo.compare_stats(h, c, "f32", tol), tol)) is expect
+        assert vo.spot_check(h[None, :], np.zeros(d, int), cols, c, eps, 0.75)[2] is expect
+
+
+def test_synthetic_weight_scale_keeps_bf16_rounding_noise_from_growing():
+    """Input recipe evidence: at d_model = 4096 a plain N(0, 0.02) initialisation gives every projection a gain of
+    0.02 * sqrt(4096) = 1.28, and such a random network amplifies bf16 rounding noise from block to block; with the
+    constant-gain scale 0.02 * sqrt(256 / d_model) it does not.  Measured on the oracle alone: its bf16-emulating
+    decode against its own float64 prefill, 16 tokens, 3 blocks of width 4096 (narrow FFN to keep this quick)."""
+    shape = synth.ModelShape(3, 4096, 8, 2, 128, 1024, 64, 500000.0)
+    tokens = np.arange(16) % shape.vocab
+
+    def drift(std):
+        rng = np.random.default_rng(3)
+        r = lambda *s: rng.standard_normal(s) * std
+        layers = [{"attn_norm": 1 + 0.1 * rng.standard_normal(shape.d_model), "wq": r(shape.d_q, shape.d_model),
+                   "wk": r(shape.d_kv, shape.d_model), "wv": r(shape.d_kv, shape.d_model), "wo": r(shape.d_model, shape.d_q),
+                   "ffn_norm": 1 + 0.1 * rng.standard_normal(shape.d_model), "w_gate": r(shape.d_ffn, shape.d_model),
+                   "w_up": r(shape.d_ffn, shape.d_model), "w_down": r(shape.d_model, shape.d_ffn)}
+                  for _ in range(shape.n_layers)]
+        layers = [{k: vo.round_to_bf16(v) for k, v in lw.items()} for lw in layers]
+        m = vo.make_model(shape, vo.round_to_bf16(rng.standard_normal((shape.vocab, shape.d_model)) * 0.02),
+                          np.ones(shape.d_model), layers)
+        exact = vo.forward_prefill(m, tokens)
+        emul = vo.forward_decode_kvcache(m, tokens, "bf16")
+        rel = np.linalg.norm(emul - exact, axis=-1) / np.linalg.norm(exact, axis=-1)  # [layers, tokens]
+        return rel.max(axis=1)
+
+    plain = drift(0.02)
+    scaled = drift(synth.weight_std(shape))
+    assert synth.weight_std(shape) == 0.02 * (256 / 4096) ** 0.5
+    assert np.all(np.diff(plain) > 0) and plain[-1] > 2 * scaled[-1], (plain, scaled)
+    assert scaled.max() <= 5e-3, scaled
+    assert plain[-1] >= 8e-3, plain
