@@ -442,11 +442,15 @@ def selftest_wait_timeout(limit_cycles: int, device="cuda:0", stream: Optional[t
     return status, gave_up
 
 
-def merkle_roots(states: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
-    """states float32 device [n_vec][d] -> uint8 device [n_vec][32] SHA-256 Merkle roots over float32 leaves."""
+def merkle_roots(states: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
+                 out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """states float32 device [n_vec][d] -> uint8 device [n_vec][32] SHA-256 Merkle roots over float32 leaves
+    (written to `out` if given)."""
     if states.dtype != torch.float32 or not states.is_contiguous() or states.dim() != 2:
         raise ValueError("states must be a contiguous float32 matrix")
-    roots = torch.empty(states.shape[0], 32, dtype=torch.uint8, device=states.device)
+    roots = out if out is not None else torch.empty(states.shape[0], 32, dtype=torch.uint8, device=states.device)
+    if roots.dtype != torch.uint8 or tuple(roots.shape) != (states.shape[0], 32) or not roots.is_contiguous():
+        raise ValueError("out must be a contiguous uint8 [n_vec][32] tensor")
     with torch.cuda.device(states.device):
         _check(lib().verillm_merkle_roots(states.data_ptr(), states.shape[0], states.shape[1], roots.data_ptr(),
                                           _stream_ptr(stream)), "verillm_merkle_roots")

@@ -63,6 +63,13 @@ struct CmpAcc {
         ss = rr = sa = sg = mx = 0.f;
         n_mis = n_large_m = n_small_w = n_exact = n_qsmall = n_zlarge = n_nonfinite = 0u;
     }
+    // Adds what a CmpPairAcc gathered (sums of the even and odd elements, in that order).
+    __device__ __forceinline__ void fold(const float2 ss2, const float2 rr2, const float2 sg2, const float2 sa2) {
+        ss += ss2.x + ss2.y;
+        rr += rr2.x + rr2.y;
+        sg += sg2.x + sg2.y;
+        sa += sa2.x + sa2.y;
+    }
 
     // h: recomputed value (fp32); hb: h rounded to the commit dtype, as a float32 bit pattern; cb: the
     // committed value as a float32 bit pattern (a bf16 value widened by 16 zero bits, or the float32).
@@ -116,6 +123,56 @@ struct CmpAcc {
         const uint32_t h_pair = pack_bf16(h_lo, h_hi);
         add_bits<kChecked>(h_lo, h_pair << 16, c_pair << 16, p);
         add_bits<kChecked>(h_hi, h_pair & 0xFFFF0000u, c_pair & 0xFFFF0000u, p);
+    }
+    // The same two elements without the test for non-finite operands, on the packed words: the float sums run on
+    // packed fp32 pairs (the caller owns the four pair accumulators and folds them in at the end), the field tests
+    // on the two 16-bit halves in place.  Counts are identical to add_bits'; the sums differ only in their order.
+    __device__ __forceinline__ void add_bf16x2_packed(float h_lo, float h_hi, uint32_t c_pair, const CmpParams& p,
+                                                      float2& ss2, float2& rr2, float2& sg2, float2& sa2) {
+        const uint32_t h_pair = pack_bf16(h_lo, h_hi);
+        const float2 c2 = make_float2(__uint_as_float(c_pair << 16), __uint_as_float(c_pair & 0xFFFF0000u));
+        const float2 d2 = cmp_ffma2(c2, make_float2(-1.f, -1.f), make_float2(h_lo, h_hi));  // h - c, exactly
+        ss2 = cmp_ffma2(d2, d2, ss2);
+        rr2 = cmp_ffma2(c2, c2, rr2);
+        sg2 = cmp_fadd2(sg2, d2);
+        const float a0 = fabsf(d2.x), a1 = fabsf(d2.y);
+        sa2.x += a0;
+        sa2.y += a1;
+        mx = fmaxf(mx, fmaxf(a0, a1));
+        n_qsmall += (a0 <= 1e-5f) ? 1u : 0u;
+        n_qsmall += (a1 <= 1e-5f) ? 1u : 0u;
+        n_zlarge += (a0 > p.tau_large) ? 1u : 0u;
+        n_zlarge += (a1 > p.tau_large) ? 1u : 0u;
+
+        const uint32_t x = h_pair ^ c_pair;
+        // low half: fields at bits 15 / 14..7 / 6..0, distances in units of 1 (thresholds scaled down by 2^16)
+        {
+            const bool same_exp = (x & 0x7F80u) == 0u;
+            const uint32_t mh = h_pair & 0x7Fu, mc = c_pair & 0x7Fu;
+            int dev = static_cast<int>(__usad(mh, mc, 0u));
+            n_mis += same_exp ? 0u : 1u;
+            n_large_m += (!same_exp && dev > (p.thr_em >> 16)) ? 1u : 0u;
+            if (same_exp && (x & 0x8000u) != 0u) {
+                const uint32_t one = (h_pair & 0x7F80u) != 0u ? 0x80u : 0u;
+                dev = static_cast<int>(mh + mc + 2u * one);
+            }
+            n_small_w += (same_exp && dev <= (p.thr_dev >> 16)) ? 1u : 0u;
+            n_exact += ((x & 0xFFFFu) == 0u) ? 1u : 0u;
+        }
+        // high half: the same fields 16 bits up, distances in the units of the float32 bit pattern
+        {
+            const bool same_exp = (x & 0x7F800000u) == 0u;
+            const uint32_t mh = h_pair & 0x7F0000u, mc = c_pair & 0x7F0000u;
+            int dev = static_cast<int>(__usad(mh, mc, 0u));
+            n_mis += same_exp ? 0u : 1u;
+            n_large_m += (!same_exp && dev > p.thr_em) ? 1u : 0u;
+            if (same_exp && static_cast<int>(x) < 0) {
+                const uint32_t one = (h_pair & 0x7F800000u) != 0u ? 0x800000u : 0u;
+                dev = static_cast<int>(mh + mc + 2u * one);
+            }
+            n_small_w += (same_exp && dev <= p.thr_dev) ? 1u : 0u;
+            n_exact += ((x & 0xFFFF0000u) == 0u) ? 1u : 0u;
+        }
     }
     template <bool kChecked = true>
     __device__ __forceinline__ void add_f32(float h, uint32_t c_bits, const CmpParams& p) {

@@ -125,14 +125,28 @@ __device__ __forceinline__ void compare_row_pass(CmpAcc& a, const float* __restr
                                                  size_t row, int d, int lane, const CmpParams& cmp) {
     if (cmp.commit_dtype == VERILLM_BF16) {
         const uint4* c4 = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(committed) + row * d);
-        for (int j = lane * 8; j < d; j += 256) {
-            const uint4 cv = __ldg(c4 + j / 8);
-            const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
-            const float4 h1 = __ldg(reinterpret_cast<const float4*>(h + j + 4));
-            a.add_bf16x2<kChecked>(h0.x, h0.y, cv.x, cmp);
-            a.add_bf16x2<kChecked>(h0.z, h0.w, cv.y, cmp);
-            a.add_bf16x2<kChecked>(h1.x, h1.y, cv.z, cmp);
-            a.add_bf16x2<kChecked>(h1.z, h1.w, cv.w, cmp);
+        if constexpr (kChecked) {
+            for (int j = lane * 8; j < d; j += 256) {
+                const uint4 cv = __ldg(c4 + j / 8);
+                const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
+                const float4 h1 = __ldg(reinterpret_cast<const float4*>(h + j + 4));
+                a.add_bf16x2<true>(h0.x, h0.y, cv.x, cmp);
+                a.add_bf16x2<true>(h0.z, h0.w, cv.y, cmp);
+                a.add_bf16x2<true>(h1.x, h1.y, cv.z, cmp);
+                a.add_bf16x2<true>(h1.z, h1.w, cv.w, cmp);
+            }
+        } else {
+            float2 ss2 = make_float2(0.f, 0.f), rr2 = ss2, sg2 = ss2, sa2 = ss2;
+            for (int j = lane * 8; j < d; j += 256) {
+                const uint4 cv = __ldg(c4 + j / 8);
+                const float4 h0 = __ldg(reinterpret_cast<const float4*>(h + j));
+                const float4 h1 = __ldg(reinterpret_cast<const float4*>(h + j + 4));
+                a.add_bf16x2_packed(h0.x, h0.y, cv.x, cmp, ss2, rr2, sg2, sa2);
+                a.add_bf16x2_packed(h0.z, h0.w, cv.y, cmp, ss2, rr2, sg2, sa2);
+                a.add_bf16x2_packed(h1.x, h1.y, cv.z, cmp, ss2, rr2, sg2, sa2);
+                a.add_bf16x2_packed(h1.z, h1.w, cv.w, cmp, ss2, rr2, sg2, sa2);
+            }
+            a.fold(ss2, rr2, sg2, sa2);
         }
     } else {
         const uint4* c4 = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(committed) + row * d);

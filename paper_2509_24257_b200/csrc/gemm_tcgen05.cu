@@ -796,8 +796,10 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
     constexpr bool additive = EPI == EPI_RESID_ADD || EPI == EPI_RESID_ADD_COMPARE;
     const SplitPlan plan = split_plan(num_tiles, q.pairs_total, (p.K + BK - 1) / BK, additive && p.split_flags != nullptr);
     if (plan.split > 1) {  // the per-tile part counters of the last round start at zero
-        const cudaError_t e = cudaMemsetAsync(p.split_flags, 0, sizeof(int) * plan.rem, stream);
-        if (e != cudaSuccess) return e;
+        if (!p.split_prezeroed) {
+            const cudaError_t e = cudaMemsetAsync(p.split_flags, 0, sizeof(int) * plan.rem, stream);
+            if (e != cudaSuccess) return e;
+        }
     } else {
         q.split_flags = nullptr;
     }

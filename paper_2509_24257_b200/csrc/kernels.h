@@ -63,6 +63,9 @@ struct GemmParams {
     // descriptor prefetch) runs under the tail of the kernel before it in the stream; the kernel waits for that
     // kernel's completion before it reads or writes any global memory.
     int overlap_prologue;
+    // 1: split_flags points at zeroed counters that belong to this launch alone (cleared before the chain of
+    // kernels started), so the launcher queues no clearing between the kernels.
+    int split_prezeroed;
     int* status;
 };
 

@@ -93,8 +93,8 @@ __device__ __noinline__ void hash_pair(const uint32_t* l, int ls, const uint32_t
     for (int i = 0; i < 8; ++i) out[i * os] = st[i];
 }
 
-constexpr int kMerkleThreads = 256;
-constexpr int kMerkleCtasPerSm = 4;  // a serial chain of rounds needs many warps to fill the issue slots
+constexpr int kMerkleThreads = 512;
+constexpr int kMerkleCtasPerSm = 3;  // 48 warps per SM: a serial chain of rounds needs many warps to fill the issue slots
 constexpr int kMerkleScratchWords = 2 * 8 * kMerkleThreads;  // two digests per thread, word-major
 
 __global__ void __launch_bounds__(kMerkleThreads, kMerkleCtasPerSm)

@@ -80,6 +80,10 @@ struct verillm_model {
     std::vector<int> h_cu, h_tok_of_slot, h_seq_of_slot, h_claimed;
     float* partials = nullptr;
     int* split_flags = nullptr;  // K-part counters of the GEMMs' last round (one per pair of SMs)
+    // K-part counters of the additive projections of one call, kSplitInts per launch, cleared once before the
+    // first layer: a clearing queued between two kernels would keep the later one's prologue from overlapping
+    int* split_arena = nullptr;
+    size_t split_launches = 0;  // launches the arena has room for
     float* sumsq = nullptr;  // [max_tokens][n_tiles_d]: per-tile sums of squares of the residual rows (folded RMSNorm)
     float2* rope_cs = nullptr;
     CUtensorMap t_xn, t_attn, t_mid;
@@ -206,7 +210,16 @@ struct LayerRun {
     const GemmParams* cmp_layer;  // fields slot_first .. cmp, or nullptr
     int next_layer;               // layer whose attention norm follows this block's output, -1 if none
     bool norm_ready;              // in/out: xn / sumsq already hold the input of this layer's attention norm
+    size_t split_cursor = 0;  // next free slot of the K-part counter arena
 };
+constexpr int kSplitInts = 80;  // one counter per tile of a last round (at most 73 with 74 pairs of SMs)
+
+// Clears the K-part counters of a call; to be queued before its first layer.
+int split_reset(verillm_model* m, LayerRun& r, cudaStream_t st) {
+    r.split_cursor = 0;
+    CU_TRY(cudaMemsetAsync(m->split_arena, 0, m->split_launches * kSplitInts * sizeof(int), st));
+    return VERILLM_OK;
+}
 
 int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st, int* launches) {
     const verillm_config& c = m->cfg;
@@ -219,7 +232,7 @@ int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st
     p.overlap_prologue = 1;  // the five kernels of a block chain their prologues under each other's tails
     // Tile walk in bands of 16 tile-rows for every projection (measured: bands of 4, 8, 32 and "all rows" are
     // no faster, also for the K = d_model projections whose activations would fit in L2).
-    const int band_d = 16;
+    const int band_qkv = 16, band_o = 16, band_gate_up = 16, band_down = 16;
     const bool fold = p.pair != 0;  // the coalesced residual epilogue of the CTA-pair kernel carries the producer half
     auto consumer = [&](GemmParams& q) {
         q.sumsq_in = m->sumsq; q.n_parts = m->n_tiles_d; q.norm_eps = c.rms_eps; q.norm_inv_d = 1.f / static_cast<float>(c.d_model);
@@ -227,13 +240,23 @@ int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st
     auto producer = [&](GemmParams& q, const void* gain) {
         q.norm_gain = gain; q.xg_out = gain ? m->xn : nullptr; q.sumsq_out = gain ? m->sumsq : nullptr;
     };
+    // K-part counters of an additive projection: a zeroed slot of its own where the arena has one left
+    auto split_slot = [&](GemmParams& q) {
+        if (p.pair && r.split_cursor < m->split_launches) {
+            q.split_flags = m->split_arena + (r.split_cursor++) * kSplitInts;
+            q.split_prezeroed = 1;
+        } else {
+            q.split_flags = m->split_flags;
+            q.split_prezeroed = 0;
+        }
+    };
 
     if (!r.norm_ready) {
         CU_TRY(launch_prenorm(m->resid, w.attn_norm, m->xn, m->sumsq, m->n_tiles_d, r.M, c.d_model, st));
         prof_mark(m, VERILLM_PROF_RMSNORM, st);
         *launches += 1;
     }
-    p.N = m->n_qkv; p.K = c.d_model; p.out = m->qkv; p.ldo = m->n_qkv; p.group_m = band_d;
+    p.N = m->n_qkv; p.K = c.d_model; p.out = m->qkv; p.ldo = m->n_qkv; p.group_m = band_qkv;
     p.rope_cs = m->rope_cs; p.pos_of_token = m->pos_of_token; p.head_dim = c.head_dim; p.rope_cols = m->d_q + m->d_kv;
     consumer(p);
     CU_TRY(launch_gemm(EPI_QKV_ROPE, m->t_xn, p.pair ? w.t_wqkv_h : w.t_wqkv, p, m->num_sms, st));
@@ -242,10 +265,10 @@ int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st
                                c.head_dim, m->attn, status, m->num_sms, 1, st));
     prof_mark(m, VERILLM_PROF_ATTENTION, st);
     p.N = c.d_model; p.K = m->d_q; p.out = m->resid; p.ldo = c.d_model;
-    p.group_m = band_d;
+    p.group_m = band_o;
     p.sumsq_in = nullptr;
-    p.split_flags = m->split_flags;
     producer(p, fold ? w.ffn_norm : nullptr);
+    split_slot(p);
     CU_TRY(launch_gemm(EPI_RESID_ADD, m->t_attn, p.pair ? w.t_wo_h : w.t_wo, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_O, st);
     if (!fold) {
@@ -253,16 +276,16 @@ int run_layer(verillm_model* m, int l, LayerRun& r, int* status, cudaStream_t st
         prof_mark(m, VERILLM_PROF_RMSNORM, st);
         *launches += 1;
     }
-    p.N = 2 * c.d_ffn; p.K = c.d_model; p.out = m->mid; p.ldo = c.d_ffn; p.group_m = band_d;
-    p.split_flags = nullptr;
+    p.N = 2 * c.d_ffn; p.K = c.d_model; p.out = m->mid; p.ldo = c.d_ffn; p.group_m = band_gate_up;
     producer(p, nullptr);
     consumer(p);
+    p.split_flags = nullptr;
     CU_TRY(launch_gemm(EPI_SWIGLU, m->t_xn, p.pair ? w.t_wgu_h : w.t_wgu, p, m->num_sms, st));
     prof_mark(m, VERILLM_PROF_GEMM_GATE_UP, st);
     p.N = c.d_model; p.K = c.d_ffn; p.out = m->resid; p.ldo = c.d_model;
-    p.group_m = band_d;
+    p.group_m = band_down;
     p.sumsq_in = nullptr;
-    p.split_flags = m->split_flags;
+    split_slot(p);
     const bool feeds_next = fold && r.next_layer >= 0;
     producer(p, feeds_next ? m->layers[r.next_layer].attn_norm : nullptr);
     if (r.cmp_layer) {
@@ -337,7 +360,7 @@ void verillm_free(verillm_model* m) {
     cudaFree(m->pos_of_token); cudaFree(m->seq_of_token); cudaFree(m->slot_first); cudaFree(m->slot_next);
     cudaFree(m->tok_of_slot); cudaFree(m->seq_of_slot); cudaFree(m->cu_dev); cudaFree(m->status);
     cudaFree(m->seq_flags);
-    cudaFree(m->partials); cudaFree(m->sumsq); cudaFree(m->split_flags); cudaFree(m->rope_cs);
+    cudaFree(m->partials); cudaFree(m->sumsq); cudaFree(m->split_flags); cudaFree(m->split_arena); cudaFree(m->rope_cs);
     cudaFree(m->lm_head); cudaFree(m->tm_y); cudaFree(m->tm_rec); cudaFree(m->tm_claimed);
     DecodeState& d = m->dec;
     cudaFree(d.kv_cache); cudaFree(d.hidden_tmp); cudaFree(d.resid); cudaFree(d.qkv); cudaFree(d.gu);
@@ -466,6 +489,8 @@ int verillm_load_weights(const verillm_config* cfg, const verillm_weights* weigh
     TRY_RC(dev_alloc(&m->partials, static_cast<size_t>(c.n_layers) * NC * m->n_tiles_d * kNPart));
     TRY_RC(dev_alloc(&m->sumsq, T * m->n_tiles_d));
     TRY_RC(dev_alloc(&m->split_flags, 256));
+    m->split_launches = static_cast<size_t>(c.n_layers) * 2;
+    TRY_RC(dev_alloc(&m->split_arena, m->split_launches * kSplitInts));
     cudaMemset(m->split_flags, 0, 256 * sizeof(int));
     TRY_RC(dev_alloc(&m->rope_cs, T * (c.head_dim / 2)));
 
@@ -584,6 +609,7 @@ static int verify_impl(verillm_model* m, const int32_t* tokens, const void* stat
     cl.slot_first = m->slot_first; cl.slot_next = m->slot_next; cl.n_check = n_check;
     cl.cmp = cmp_params(*tol, commit_dtype);
     LayerRun run{M, batch, max_len, m->cu_dev, n_check > 0 ? &cl : nullptr, -1, false};
+    if ((rc = split_reset(m, run, st))) return rc;
     for (int l = l0; l < l1; ++l) {
         run.next_layer = l + 1 < l1 ? l + 1 : -1;
         const size_t slab = static_cast<size_t>(l - l0) * n_check;
@@ -857,6 +883,7 @@ int verillm_decode_commit(verillm_model* m, const int32_t* tokens, const int32_t
         cl.committed = nullptr; cl.partials = nullptr;
         LayerRun run{Mp, batch, max_np, m->cu_dev, n_check > 0 ? &cl : nullptr, -1, false};
         int launches = 0;
+        if ((rc = split_reset(m, run, st))) return rc;
         for (int l = 0; l < c.n_layers; ++l) {
             run.next_layer = l + 1 < c.n_layers ? l + 1 : -1;
             cl.hidden_out = d.hidden_tmp + static_cast<size_t>(l) * n_check * c.d_model;
