@@ -34,8 +34,11 @@ TOL_REL_L2 = 5e-2
 # x 10, 8 final adds), and the average the Merkle kernel executes per compression of a 4096-entry tree (profiler
 # instruction count: the padding block of every inner node has a constant schedule, most of a leaf's folds away)
 SHA256_INT_OPS = 64 * 14 + 48 * 10 + 8
-SHA256_INT_OPS_EXECUTED = 1276
-GATE_UP_DRAM_BYTES_8B = 657.4e6 + 225.3e6  # measured, per launch, M = 8192 tokens at the 8B widths
+SHA256_INT_OPS_EXECUTED = 1286
+# of which funnel shifts (rotations): 6 per round everywhere, 4 per schedule word where a schedule is computed
+# (all 48 words of an inner node's first block, about a third of a leaf's): about 490 on average
+SHA256_FUNNEL_SHIFTS_EXECUTED = 490
+GATE_UP_DRAM_BYTES_8B = 668.7e6 + 227.9e6  # measured, per launch, M = 8192 tokens at the 8B widths
 
 
 def measured_peaks():
@@ -343,6 +346,36 @@ def bench_full_coverage(model, wl, flat, cu, tol, device, stream, peaks, down_ms
             "positions_accepted": int((res["pos_ok"] == 1).sum()), "status": res["status"]}
 
 
+def bench_merkle(n_vec, d_model, device, stream, clocks, iters: int = 10):
+    """Merkle commitment of n_vec state vectors (one SHA-256 tree per (layer, position) vector): integer ALU work."""
+    import torch
+    from paper_2509_24257_b200 import binding as vb
+
+    mk_in = torch.randn(n_vec, d_model, device=device)
+    mk_out = torch.empty(mk_in.shape[0], 32, dtype=torch.uint8, device=device)
+    mk_ms = timed_light(lambda: vb.merkle_roots(mk_in, stream, out=mk_out), stream, iters)
+    n_compress = mk_in.shape[0] * (4 * ((d_model + 1) // 2) + 2 * ((d_model + 1) // 2 - 1))
+    # ALU peak: one SHA-256 compression is 1384 32-bit integer instructions as written (64 rounds x 14, 48 schedule
+    # words x 10, 8 final adds); an SM issues 4 warp instructions = 128 lane operations per clock
+    props = torch.cuda.get_device_properties(device)
+    sm_clock_hz = 1e6 * float(clocks.get("sm_max_mhz") or 1965.0)
+    lane_ops_peak = props.multi_processor_count * 128 * sm_clock_hz
+    mk_peak = lane_ops_peak / SHA256_INT_OPS
+    mk_rate = n_compress / (mk_ms * 1e-3)
+    # funnel shifts (every rotation: 6 of a round's 14 instructions, 4 of a schedule word's 10) issue at half
+    # rate on this part (64 lanes per clock per SM, measured), so a full-rate count overstates what the ALUs can do
+    merkle = {"vectors": int(mk_in.shape[0]), "scalars_per_vector": d_model, "ms": round(mk_ms, 4), "bound": "alu",
+              "ns_per_scalar": round(mk_ms * 1e6 / mk_in.numel(), 4),
+              "sha256_compressions_per_s": round(mk_rate, 0), "peak_compressions_per_s": round(mk_peak, 0),
+              "frac": round(mk_rate / mk_peak, 4),
+              "peak_kind": "derived: SMs x 128 integer lane-ops per clock x max SM clock / 1384 ops per full compression",
+              "ops_executed_per_compression": SHA256_INT_OPS_EXECUTED,
+              "frac_of_lane_op_peak_executed": round(mk_rate * SHA256_INT_OPS_EXECUTED / lane_ops_peak, 4),
+              "frac_with_half_rate_rotations": round(
+                  mk_rate * (SHA256_INT_OPS_EXECUTED + SHA256_FUNNEL_SHIFTS_EXECUTED) / lane_ops_peak, 4)}
+    return merkle
+
+
 def run_compare_only(args, wl):
     """Runs only the comparison path (no model): a small process for profiler captures of its kernels."""
     import torch
@@ -354,6 +387,17 @@ def run_compare_only(args, wl):
     tol = vb.default_tol(rel_l2=TOL_REL_L2)
     print(json.dumps({"compare_path": bench_compare_path(wl, device, tol, peaks, torch.cuda.current_stream(),
                                                          iters=max(args.steps, 1))}))
+
+
+def run_merkle_only(args, wl):
+    """Runs only the Merkle commitment kernel (no model): a small process for profiler captures."""
+    import torch
+
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    n_vec = wl.shape.n_layers * max(1, int(round(wl.check_frac * wl.n_tokens)))
+    print(json.dumps({"merkle": bench_merkle(n_vec, wl.shape.d_model, device, torch.cuda.current_stream(), {},
+                                            iters=max(args.steps, 1))}))
 
 
 def run_ours(args, wl):
@@ -404,26 +448,47 @@ def run_ours(args, wl):
     value = vdist.aggregate_throughput(float(wl.n_tokens * args.steps), seconds)
     slowest = vdist.max_over_ranks(seconds)
 
-    # ---- end to end: host buffers in, report out, every step
+    # ---- end to end: host buffers in, report out, every step.  Inputs of step i + 1 are uploaded from pinned memory
+    # on a copy stream while step i computes (two device buffers); every upload, every call and every read-back of
+    # the report lies inside the timed region, and the host waits for each step's report before it goes on.
     pin = lambda t: t.cpu().pin_memory()
     tok_pin, comm_pin = pin(flat), pin(committed)
     out_pin = {k: torch.empty_like(getattr(report, k), device="cpu").pin_memory()
                for k in ("stats", "pos_ok", "first_bad_layer", "seq_ok", "seq_score", "status")}
-    tok_dev, comm_dev = torch.empty_like(flat), torch.empty_like(committed)
+    in_dev = [(torch.empty_like(flat), torch.empty_like(committed)) for _ in range(2)]
+    copy_stream = torch.cuda.Stream(device=device)
+    uploaded = [torch.cuda.Event() for _ in range(2)]
+    consumed = [torch.cuda.Event() for _ in range(2)]
 
-    def e2e_step():
-        tok_dev.copy_(tok_pin, non_blocking=True)
-        comm_dev.copy_(comm_pin, non_blocking=True)
-        model.verify_prefill(tok_dev, cu, comm_dev, cs, cp, tol, report=report, stream=stream)
-        for k, buf in out_pin.items():
-            buf.copy_(getattr(report, k), non_blocking=True)
-        torch.cuda.synchronize()
+    def upload(i):
+        tok_dev, comm_dev = in_dev[i % 2]
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(consumed[i % 2])  # the step that last read this buffer has finished with it
+            tok_dev.copy_(tok_pin, non_blocking=True)
+            comm_dev.copy_(comm_pin, non_blocking=True)
+            uploaded[i % 2].record(copy_stream)
 
-    e2e_step()
+    def e2e_run(n):
+        upload(0)
+        for i in range(n):
+            if i + 1 < n:
+                upload(i + 1)
+            tok_dev, comm_dev = in_dev[i % 2]
+            stream.wait_event(uploaded[i % 2])
+            model.verify_prefill(tok_dev, cu, comm_dev, cs, cp, tol, report=report, stream=stream)
+            consumed[i % 2].record(stream)
+            for k, buf in out_pin.items():
+                buf.copy_(getattr(report, k), non_blocking=True)
+            stream.synchronize()
+
+    for ev in consumed:
+        ev.record(stream)
+    e2e_run(2)
+    torch.cuda.synchronize()
     vdist.barrier()
     t0 = time.perf_counter()
-    for _ in range(args.steps):
-        e2e_step()
+    e2e_run(args.steps)
+    torch.cuda.synchronize()
     e2e_seconds = time.perf_counter() - t0
     vdist.barrier()
     e2e_value = vdist.aggregate_throughput(float(wl.n_tokens * args.steps), e2e_seconds)
@@ -482,29 +547,7 @@ def run_ours(args, wl):
         down_sampled = acc["gemm_down_resid_compare"][0] / acc["gemm_down_resid_compare"][1]
         full_coverage = bench_full_coverage(model, wl, flat, cu, tol, device, stream, peaks, down_sampled)
 
-    # ---- Merkle commitment of the checked states (one SHA-256 tree per (layer, position) vector): integer ALU work
-    mk_in = torch.randn(s.n_layers * len(cs), s.d_model, device=device)
-    mk_out = torch.empty(mk_in.shape[0], 32, dtype=torch.uint8, device=device)
-    mk_ms = timed_light(lambda: vb.merkle_roots(mk_in, stream, out=mk_out), stream, 10)
-    n_compress = mk_in.shape[0] * (4 * ((s.d_model + 1) // 2) + 2 * ((s.d_model + 1) // 2 - 1))
-    # ALU peak: one SHA-256 compression is 1384 32-bit integer instructions as written (64 rounds x 14, 48 schedule
-    # words x 10, 8 final adds); an SM issues 4 warp instructions = 128 lane operations per clock
-    props = torch.cuda.get_device_properties(device)
-    sm_clock_hz = 1e6 * float(clocks.get("sm_max_mhz") or 1965.0)
-    lane_ops_peak = props.multi_processor_count * 128 * sm_clock_hz
-    mk_peak = lane_ops_peak / SHA256_INT_OPS
-    mk_rate = n_compress / (mk_ms * 1e-3)
-    # funnel shifts (every rotation: 6 of a round's 14 instructions, 4 of a schedule word's 10) issue at half
-    # rate on this part (64 lanes per clock per SM, measured), so a full-rate count overstates what the ALUs can do
-    merkle = {"vectors": int(mk_in.shape[0]), "scalars_per_vector": s.d_model, "ms": round(mk_ms, 4), "bound": "alu",
-              "ns_per_scalar": round(mk_ms * 1e6 / mk_in.numel(), 4),
-              "sha256_compressions_per_s": round(mk_rate, 0), "peak_compressions_per_s": round(mk_peak, 0),
-              "frac": round(mk_rate / mk_peak, 4),
-              "peak_kind": "derived: SMs x 128 integer lane-ops per clock x max SM clock / 1384 ops per full compression",
-              "ops_executed_per_compression": SHA256_INT_OPS_EXECUTED,
-              "frac_of_lane_op_peak_executed": round(mk_rate * SHA256_INT_OPS_EXECUTED / lane_ops_peak, 4),
-              "frac_with_half_rate_rotations": round(mk_rate * (SHA256_INT_OPS + 64 * 6 + 48 * 4) / lane_ops_peak, 4)}
-    del mk_in
+    merkle = bench_merkle(s.n_layers * len(cs), s.d_model, device, stream, clocks)
 
     if rank == 0:
         run, desc = oracle_sample(wl, 12.0, str(device)) if args.gpus == 1 else (None, None)
@@ -531,7 +574,9 @@ def run_ours(args, wl):
             "verdicts": {"seq_ok": res["seq_ok"].tolist(), "positions_rejected": int((res["pos_ok"] == 0).sum()),
                          "status": res["status"]},
             "clocks": clocks, "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-                                     "d2h_bytes_per_step": int(d2h)},
+                                     "d2h_bytes_per_step": int(d2h),
+                                     "pipelining": "inputs of step i+1 are uploaded on a copy stream while step i runs; "
+                                                   "the host waits for every step's report"},
             "gpu_launches": int(launches), "roofline": roofline, "token_match": token_match, "compare_path": compare_path,
             "full_coverage": full_coverage, "merkle": merkle,
             "cpu_baseline": cpu_baseline,
@@ -550,6 +595,8 @@ def main():
     ap.add_argument("--workload", default="llama8b")
     ap.add_argument("--compare-only", action="store_true",
                     help="time only the standalone comparison path at the workload's widths (no model is built)")
+    ap.add_argument("--merkle-only", action="store_true",
+                    help="time only the Merkle commitment of the workload's checked states (no model is built)")
     ap.add_argument("--no-full-coverage", action="store_true",
                     help="skip the supplementary run that checks every position (it holds 6 GB more on the device)")
     ap.add_argument("--layers", type=int, default=0,
@@ -565,6 +612,8 @@ def main():
         run_reference(args, wl)
     elif args.compare_only:
         run_compare_only(args, wl)
+    elif args.merkle_only:
+        run_merkle_only(args, wl)
     else:
         run_ours(args, wl)
 
