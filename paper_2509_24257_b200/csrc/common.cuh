@@ -14,6 +14,7 @@ namespace vl {
 // A wait that has not completed after this many SM clock cycles (about two seconds) gives up, records
 // VERILLM_DEV_WAIT_TIMEOUT and lets the kernel run to its end, so that the context stays usable.
 constexpr long long kWaitLimitCycles = 4000000000LL;
+constexpr unsigned kWaitSuspendNs = 20000u;  // longest single suspension of a waiting thread (the hardware may cap it lower)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -48,6 +49,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// The same with a suspend-time hint: the thread may stay suspended (issuing nothing) for up to about `ns`
+// nanoseconds, and resumes when the phase completes.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
 // Non-blocking probe of a phase parity (try_wait may suspend the thread for a while; this never does).
 __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -65,12 +81,12 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait on a phase parity: gives up after `limit_cycles` SM clock cycles.  Returns false (after
 // recording the timeout in *status) if the limit ran out.
 __device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, int* status, long long limit_cycles) {
-#pragma unroll 1
-    for (int i = 0; i < 128; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
+    // A waiting thread should not compete for issue slots with the warps that do the work: let the hardware
+    // keep it suspended until the phase completes (the hint bounds one suspension, the clock the whole wait).
     const long long t0 = clock64();
 #pragma unroll 1
-    while (!mbar_try_wait(bar, parity)) {
+    while (!mbar_try_wait_hint(bar, parity, kWaitSuspendNs)) {
         if (clock64() - t0 > limit_cycles) {
             if (status) atomicCAS(status, 0, VERILLM_DEV_WAIT_TIMEOUT);
             return false;
