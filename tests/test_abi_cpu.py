@@ -3,6 +3,7 @@ arguments before touching a device, and the multi-process replica plumbing works
 import ctypes
 import os
 import re
+import sys
 
 import pytest
 
@@ -107,3 +108,23 @@ def test_workload_table_matches_the_stated_configs():
     assert tuple(w[n].n_check for n in names) == (64, 20, 82, 41, 20)
     assert abs(w["llama8b"].total_flops() / 1e12 - 116.6) < 0.2 and abs(w["llama70b"].total_flops() / 1e12 - 285.9) < 0.5
     assert abs(w["llama8b"].shape.n_params() / 1e9 - 7.505) < 0.01  # embedding + 32 blocks, no output head
+
+
+def test_reference_arm_prints_the_contract_line():
+    """`bench.py --impl reference` times the oracle on the host cores and prints one JSON line with the same metric,
+    unit and workload keys as the GPU arm, `impl`, a `cpu_baseline` describing the run and an `e2e` block without copies."""
+    import json
+    import subprocess
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                          "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=300, cwd=root)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["metric"] == "verified_tokens_per_sec" and d["unit"] == "tokens/s"
+    assert d["higher_is_better"] is True and d["vs_baseline"] is None and d["dtype"] == "f64" and d["gpu_launches"] == 0
+    assert d["config"]["workload"] == "tiny" and d["value"] > 0 and d["steps"] == 1
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] == d["value"] and d["cpu_baseline"]["cores"] >= 1
+    assert d["e2e"] == {"value": d["value"], "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
